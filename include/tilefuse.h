@@ -1,0 +1,198 @@
+/*
+ * tilefuse.h -- C ABI of libtilefuse.so: the fused mixed-precision linear layer
+ *
+ *     Y[M,N] = A[M,K] . dequant(Wq)[K,N]
+ *
+ * for NVIDIA B200 (sm_100a).  Weights stay 4-bit / 8-bit in device memory and are
+ * unpacked, dequantized and multiplied inside one kernel; no bf16 copy of the weights
+ * is ever written to global memory (the fusion property of Section 4.1 of the paper).
+ *
+ * Conventions for every entry point
+ *   - "host" / "device" on a pointer says which memory it must point into.
+ *   - The caller owns every buffer.  The library allocates nothing, frees nothing and
+ *     keeps no pointer after a call returns.
+ *   - Device calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*;
+ *     NULL = the default stream) and never synchronise, except tf_device_status.
+ *   - Errors are return codes.  Nothing is printed, nothing aborts, no exception
+ *     crosses the boundary.  On any error the outputs are left untouched.
+ *   - Device pointers must be 16-byte aligned (TF_ERR_ALIGN otherwise).
+ *   - Outputs must not overlap inputs or the workspace.
+ *   - Same inputs give bit-identical outputs (no atomics on results).
+ *   - There is no CPU or other-GPU fallback: a device that is not compute capability
+ *     10.x gives TF_ERR_ARCH.
+ */
+#ifndef TILEFUSE_H
+#define TILEFUSE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum tf_status {
+    TF_OK = 0,
+    TF_ERR_NULL = 1,       /* a required pointer is NULL */
+    TF_ERR_SHAPE = 2,      /* M, K, N or group_size outside the legal set (see each call) */
+    TF_ERR_ALIGN = 3,      /* a device pointer is not 16-byte aligned */
+    TF_ERR_BLOB = 4,       /* packed blob: bad magic / version, or bits, K, N do not match */
+    TF_ERR_WORKSPACE = 5,  /* workspace missing or smaller than tf_workspace_size() */
+    TF_ERR_ARCH = 6,       /* current device is not compute capability 10.x */
+    TF_ERR_CUDA = 7,       /* a CUDA runtime call or a kernel launch failed */
+    TF_ERR_TIMEOUT = 8     /* a bounded device-side wait gave up (see tf_device_status) */
+} tf_status;
+
+/* Operation selector for tf_workspace_size. */
+typedef enum tf_op {
+    TF_OP_GEMV_W4A16 = 0,
+    TF_OP_GEMV_W8A16 = 1,
+    TF_OP_GEMM_W4A16 = 2,
+    TF_OP_GEMM_W8A16 = 3
+} tf_op;
+
+/* Limits of the problem statement (Section 2.1: C = A x B; Section 4.2: K, N up to 32K). */
+#define TF_MAX_DIM      32768   /* K and N */
+#define TF_MAX_M_GEMV   16
+#define TF_MAX_M_GEMM   4096
+#define TF_TILE_K       128     /* k-extent of one packed tile = the AWQ group size */
+#define TF_TILE_N       64      /* n-extent of one packed tile (a "strip" of columns) */
+
+/*
+ * The packed blob (output of tf_pack_awq / tf_pack_w8).
+ *
+ * Offline pre-tiling with per-tile metadata (Section 4.2): the weight matrix is cut into
+ * tiles of TF_TILE_K rows (k) x TF_TILE_N columns (n); each tile is one contiguous payload
+ * that carries its packed weights followed by the scales (and zero points) that dequantize
+ * it, so that one stream delivers everything a tile needs.  Tiles of one column strip are
+ * consecutive along K (tile-major order: a strip is one long contiguous read).
+ *
+ *   blob   = header (256 bytes) | tile(strip 0, ktile 0) | tile(0,1) | ... | tile(1,0) | ...
+ *   W4 tile (4256 bytes) = 4096 B weights | 64 fp16 scales (128 B) | 64 4-bit zeros (32 B)
+ *   W8 tile (8320 bytes) = 8192 B weights | 64 fp16 scales (128 B)
+ *
+ * Inside a tile the weights are stored in the register order of the tensor-core operand
+ * that consumes them; tf_unpack_w4 / tf_unpack_w8 are the authoritative decoders.  N is
+ * padded up to a multiple of TF_TILE_N with weights that dequantize to exactly 0
+ * (q = z, s = 0), the padding noted in Section 5.2; padded columns are never written to Y.
+ * The blob is position independent: copy it to the device with any memcpy.
+ */
+typedef struct tf_blob_header {
+    uint32_t magic;        /* 0x31424654 = "TFB1" */
+    uint32_t version;      /* 1 */
+    uint32_t bits;         /* 4 or 8 */
+    uint32_t K;
+    uint32_t N;
+    uint32_t group_size;   /* as given to the packer; a multiple of TF_TILE_K */
+    uint32_t n_padded;     /* N rounded up to a multiple of TF_TILE_N */
+    uint32_t strips;       /* n_padded / TF_TILE_N */
+    uint32_t ktiles;       /* K / TF_TILE_K */
+    uint32_t tile_bytes;   /* 4256 (W4) or 8320 (W8) */
+    uint64_t tiles_offset; /* 256 */
+    uint64_t total_bytes;  /* = tf_packed_size(bits, K, N, group_size) */
+    uint8_t  reserved[200];
+} tf_blob_header;
+
+/* Bytes of the packed blob, or 0 if the shape is illegal.
+ * Legal: bits in {4, 8}; 128 <= K <= TF_MAX_DIM; 8 <= N <= TF_MAX_DIM; N % 8 == 0;
+ * group_size % 128 == 0; K % group_size == 0. */
+size_t tf_packed_size(int bits, int K, int N, int group_size);
+
+/*
+ * Offline pre-tiling of AWQ-format W4A16 weights (Section 4.2; format of Section 2.2).
+ *   qweight     host, uint32 [K][N/8]: eight 4-bit codes per word along N; bits [4i,4i+4) of
+ *               word j hold column 8j + (0,2,4,6,1,3,5,7)[i].
+ *   scales_fp16 host, IEEE fp16 bit patterns [K/group_size][N].
+ *   qzeros      host, uint32 [K/group_size][N/8], same nibble order as qweight.
+ *   out         host, out_bytes >= tf_packed_size(4, K, N, group_size); written completely.
+ * Dequantization meaning of the result: w[k][n] = s[k/g][n] * (q[k][n] - z[k/g][n])  (Eq. 2).
+ * Pure host code, deterministic, no allocation proportional to the input.
+ * Errors: TF_ERR_NULL, TF_ERR_SHAPE (see tf_packed_size), TF_ERR_WORKSPACE (out_bytes too small).
+ */
+tf_status tf_pack_awq(const uint32_t* qweight, const uint16_t* scales_fp16, const uint32_t* qzeros,
+                      int K, int N, int group_size, void* out, size_t out_bytes);
+
+/*
+ * Offline pre-tiling of symmetric W8A16 weights (Section 4.2, last paragraph; Eq. 1).
+ *   w           host, int8 [K][N] row-major (the full range -128..127 is accepted).
+ *   scales_fp16 host, fp16 bit patterns [K/group_size][N]; group_size == K is the
+ *               per-channel case of Section 2.2.
+ * Meaning: w_hat[k][n] = s[k/g][n] * w[k][n].  Otherwise as tf_pack_awq.
+ */
+tf_status tf_pack_w8(const int8_t* w, const uint16_t* scales_fp16,
+                     int K, int N, int group_size, void* out, size_t out_bytes);
+
+/*
+ * Decode a packed blob on the GPU with the same device routines the GEMV / GEMM kernels use
+ * (the unpack step of Section 4.3).  Outputs are bit-exact copies of what was packed:
+ *   q      device, uint8 [K][N] (W4: 0..15) / int8 [K][N] (W8)
+ *   z      device, uint8 [K/group_size][N]            (W4 only)
+ *   s_fp16 device, fp16 bit patterns [K/group_size][N]
+ * Any of the output pointers may be NULL to skip that output.
+ * Errors: TF_ERR_NULL (packed), TF_ERR_SHAPE, TF_ERR_ALIGN (packed), TF_ERR_ARCH, TF_ERR_CUDA.
+ * A blob whose header does not match (bits, K, N) leaves the outputs untouched.
+ */
+tf_status tf_unpack_w4(const void* packed, uint8_t* q, uint8_t* z, uint16_t* s_fp16,
+                       int K, int N, int group_size, void* cuda_stream);
+tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s_fp16,
+                       int K, int N, int group_size, void* cuda_stream);
+
+/*
+ * Decode-phase fused GEMV (Sections 4.3 "GEMV microkernel" and 4.4): 1 <= M <= 16 tokens.
+ *   packed   device, blob from tf_pack_awq (w4a16) / tf_pack_w8 (w8a16) for this K, N.
+ *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.
+ *   y_bf16   device, bf16 [M][N] row-major, leading dimension N; fully overwritten.
+ *   workspace, workspace_bytes   device scratch of at least tf_workspace_size(op, M, K, N)
+ *            bytes (may be NULL / 0 when that size is 0).  Its first 16 bytes, when present,
+ *            receive the device status word read by tf_device_status.
+ * Arithmetic: weights are kept exact ((q - z) as small integers, scale applied in fp32 to
+ * per-group partial sums), fp32 accumulation, one round-to-nearest-even to bf16 at the end.
+ * Each CTA cluster owns a set of output columns for all K: no cross-cluster reduction.
+ * Errors: TF_ERR_NULL, TF_ERR_SHAPE (M outside 1..16, K % 128, N % 8, limits), TF_ERR_ALIGN,
+ *         TF_ERR_WORKSPACE, TF_ERR_ARCH, TF_ERR_CUDA.  A blob/argument mismatch is detected on
+ *         the device: y is left untouched and the status word (if a workspace was given)
+ *         becomes TF_ERR_BLOB.
+ */
+tf_status tf_gemv_w4a16(const void* packed, const void* a_bf16, void* y_bf16,
+                        int M, int K, int N, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+tf_status tf_gemv_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
+                        int M, int K, int N, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+
+/*
+ * Prefill-phase fused GEMM (Section 4.3 "GEMM microkernel"): 1 <= M <= 4096 tokens,
+ * K, N <= 32768.  Same arguments as the GEMV.  Each packed weight tile is dequantized once
+ * into shared memory as bf16 and reused by every token row of the CTA tile (the
+ * dequantize-once rule of Section 4.1), then multiplied on the tcgen05 tensor cores with
+ * fp32 accumulation in tensor memory.  Weights are rounded to bf16 once: w = bf16((q-z)*s).
+ * Split-K partial sums (large K, few tiles) go through the workspace.
+ * Errors as for the GEMV; M range 1..4096; a workspace of tf_workspace_size() bytes is
+ * always required (it holds at least the status word).
+ */
+tf_status tf_gemm_w4a16(const void* packed, const void* a_bf16, void* y_bf16,
+                        int M, int K, int N, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
+                        int M, int K, int N, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+
+/* Scratch bytes the given operation needs for this shape (0 if none; 0 also if the shape
+ * is illegal -- the compute call then reports TF_ERR_SHAPE). */
+size_t tf_workspace_size(int op, int M, int K, int N);
+
+/* Synchronise `cuda_stream`, read the status word at the start of `workspace` (device) and
+ * return it: TF_OK, TF_ERR_BLOB or TF_ERR_TIMEOUT; TF_ERR_CUDA if the stream reports an error.
+ * The word is sticky until the caller clears the first 16 bytes of the workspace. */
+tf_status tf_device_status(const void* workspace, void* cuda_stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char* tf_status_string(tf_status status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int tf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TILEFUSE_H */

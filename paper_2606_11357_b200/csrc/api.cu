@@ -1,0 +1,161 @@
+// C-ABI entry points: argument validation and kernel launches.  No allocation, no retained state
+// other than a per-device cache of immutable device attributes.
+#include <cuda_runtime.h>
+
+#include "../../include/tilefuse.h"
+#include "kernels.h"
+#include "layout.h"
+
+namespace {
+
+struct DeviceInfo {
+    int known;      // 0 = not queried, 1 = ok (cc 10.x), -1 = wrong architecture, -2 = query failed
+    int sm_count;
+};
+DeviceInfo g_devices[64];
+
+// Device attributes of the current device (cached after the first call on that device).
+tf_status device_info(DeviceInfo* out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return TF_ERR_CUDA;
+    DeviceInfo& d = g_devices[dev];
+    if (d.known == 0) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return TF_ERR_CUDA;
+        }
+        d.sm_count = sms;
+        d.known = major == 10 ? 1 : -1;
+    }
+    if (d.known != 1) return TF_ERR_ARCH;
+    *out = d;
+    return TF_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+tf_status check_linear_args(int bits, const void* packed, const void* a, void* y, int M, int K, int N,
+                            int max_m) {
+    if (!packed || !a || !y) return TF_ERR_NULL;
+    if (M < 1 || M > max_m) return TF_ERR_SHAPE;
+    if (tf_packed_size(bits, K, N, tf::kTileK) == 0) return TF_ERR_SHAPE;
+    if (!aligned16(packed) || !aligned16(a) || !aligned16(y)) return TF_ERR_ALIGN;
+    return TF_OK;
+}
+
+tf_status gemv(int bits, const void* packed, const void* a, void* y, int M, int K, int N, void* workspace,
+               size_t workspace_bytes, void* stream) {
+    tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMV);
+    if (st != TF_OK) return st;
+    if (workspace != nullptr && (!aligned16(workspace) || workspace_bytes < sizeof(uint32_t) * 4))
+        return workspace_bytes < 16 ? TF_ERR_WORKSPACE : TF_ERR_ALIGN;
+    DeviceInfo dev;
+    st = device_info(&dev);
+    if (st != TF_OK) return st;
+    const tf::GemvPlan plan = tf::plan_gemv(K, N, dev.sm_count);
+    cudaError_t e = tf::launch_gemv(bits, plan, packed, a, y, M, K, N, workspace, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    return TF_OK;
+}
+
+tf_status gemm(int bits, const void* packed, const void* a, void* y, int M, int K, int N, void* workspace,
+               size_t workspace_bytes, void* stream) {
+    tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMM);
+    if (st != TF_OK) return st;
+    const size_t need = tf_workspace_size(bits == 4 ? TF_OP_GEMM_W4A16 : TF_OP_GEMM_W8A16, M, K, N);
+    if (workspace == nullptr || workspace_bytes < need) return TF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return TF_ERR_ALIGN;
+    DeviceInfo dev;
+    st = device_info(&dev);
+    if (st != TF_OK) return st;
+    cudaError_t e = tf::launch_gemm(bits, packed, a, y, M, K, N, workspace, workspace_bytes, dev.sm_count,
+                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    return TF_OK;
+}
+
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_w4a16(const void* packed, const void* a, void* y, int M, int K, int N,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    return gemv(4, packed, a, y, M, K, N, workspace, workspace_bytes, stream);
+}
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_w8a16(const void* packed, const void* a, void* y, int M, int K, int N,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    return gemv(8, packed, a, y, M, K, N, workspace, workspace_bytes, stream);
+}
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_w4a16(const void* packed, const void* a, void* y, int M, int K, int N,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    return gemm(4, packed, a, y, M, K, N, workspace, workspace_bytes, stream);
+}
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_w8a16(const void* packed, const void* a, void* y, int M, int K, int N,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    return gemm(8, packed, a, y, M, K, N, workspace, workspace_bytes, stream);
+}
+
+extern "C" __attribute__((visibility("default"))) size_t tf_workspace_size(int op, int M, int K, int N) {
+    const int bits = (op == TF_OP_GEMV_W4A16 || op == TF_OP_GEMM_W4A16) ? 4 : 8;
+    if (op < TF_OP_GEMV_W4A16 || op > TF_OP_GEMM_W8A16) return 0;
+    if (tf_packed_size(bits, K, N, tf::kTileK) == 0) return 0;
+    if (op == TF_OP_GEMV_W4A16 || op == TF_OP_GEMV_W8A16) return 0;
+    if (M < 1 || M > TF_MAX_M_GEMM) return 0;
+    return tf::gemm_workspace_bytes(M, K, N);
+}
+
+static tf_status unpack_common(int bits, const void* packed, void* q, void* z, uint16_t* s, int K, int N,
+                               int group_size, void* stream) {
+    if (!packed) return TF_ERR_NULL;
+    if (tf_packed_size(bits, K, N, group_size) == 0) return TF_ERR_SHAPE;
+    if (!aligned16(packed)) return TF_ERR_ALIGN;
+    DeviceInfo dev;
+    tf_status st = device_info(&dev);
+    if (st != TF_OK) return st;
+    cudaError_t e = bits == 4
+        ? tf::launch_unpack_w4(packed, static_cast<uint8_t*>(q), static_cast<uint8_t*>(z), s, K, N, group_size,
+                               static_cast<cudaStream_t>(stream))
+        : tf::launch_unpack_w8(packed, static_cast<int8_t*>(q), s, K, N, group_size,
+                               static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    return TF_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_unpack_w4(const void* packed, uint8_t* q, uint8_t* z, uint16_t* s, int K, int N,
+                                  int group_size, void* stream) {
+    return unpack_common(4, packed, q, z, s, K, N, group_size, stream);
+}
+extern "C" __attribute__((visibility("default"))) tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s, int K, int N, int group_size,
+                                  void* stream) {
+    return unpack_common(8, packed, q, nullptr, s, K, N, group_size, stream);
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_device_status(const void* workspace, void* stream) {
+    if (!workspace) return TF_ERR_NULL;
+    uint32_t word[4] = {0, 0, 0, 0};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return TF_ERR_CUDA;
+    }
+    return word[0] <= TF_ERR_TIMEOUT ? static_cast<tf_status>(word[0]) : TF_ERR_CUDA;
+}
+
+extern "C" __attribute__((visibility("default"))) const char* tf_status_string(tf_status status) {
+    switch (status) {
+        case TF_OK: return "ok";
+        case TF_ERR_NULL: return "a required pointer is NULL";
+        case TF_ERR_SHAPE: return "illegal M, K, N or group size";
+        case TF_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case TF_ERR_BLOB: return "packed blob header does not match the arguments";
+        case TF_ERR_WORKSPACE: return "workspace or output buffer too small";
+        case TF_ERR_ARCH: return "device is not compute capability 10.x (B200)";
+        case TF_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
+        case TF_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    }
+    return "unknown status";
+}
+
+extern "C" __attribute__((visibility("default"))) int tf_version(void) { return 100; }

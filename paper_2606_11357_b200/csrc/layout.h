@@ -1,0 +1,38 @@
+// Tile layout of the packed blob, shared by the host packer and the device kernels.
+//
+// A tile covers TF_TILE_K = 128 rows (k) x TF_TILE_N = 64 columns (n).  Its weights are stored
+// in the register order of the warp-level tensor-core operand "A" of shape 16 (n) x 16 (k):
+// lane L = (g << 2) | t  (g = 0..7, t = 0..3) owns, per 16x16 block, four bf16x2 registers
+//     r0 = (row g,   k-slots 2t,2t+1)      r1 = (row g+8, k-slots 2t,2t+1)
+//     r2 = (row g,   k-slots 2t+8,2t+9)    r3 = (row g+8, k-slots 2t+8,2t+9)
+// A tile has 8 k-blocks (kb) x 4 n-blocks (w).  The contraction index may be permuted freely as
+// long as weights and activations agree, so k-slots map to physical k such that one lane reads
+// 16 consecutive activations for four consecutive k-blocks:
+//     k = k0 + 64*(kb>>2) + 16*t + 4*(kb&3) + {0,1 (r0/r1 lo,hi), 2,3 (r2/r3 lo,hi)}
+//     n = n0 + 16*w + g + 8*(register is r1 or r3)
+//
+// W4: one uint32 per (kb, lane, w) at word index (kb*32 + lane)*4 + w; nibble p holds register
+//     (p & 3), element (p >> 2)  -- so  (x >> 4*i) & 0x000F000F  is register i as two integers.
+// W8: two uint32 per (kb, lane, w): 16-byte vector (kb*2 + (w>>1))*32 + lane, words 2*(w&1)+r;
+//     byte b of word r holds register 2r + (b>>1), element (b & 1).
+// Scales: fp16 [g][2w+h] for column n0 + 16w + g + 8h  (one 16-byte vector per g).
+// Zeros (W4): uint32 [g]; nibble i (0..3) = column n0 + 16i + g, nibble i+4 = column n0+16i+g+8.
+#pragma once
+#include <stdint.h>
+
+namespace tf {
+
+constexpr int kTileK = 128;
+constexpr int kTileN = 64;
+constexpr int kHeaderBytes = 256;
+constexpr uint32_t kMagic = 0x31424654u;   // "TFB1"
+constexpr uint32_t kBlobVersion = 1;
+
+constexpr int kW4WeightBytes = 4096;
+constexpr int kW8WeightBytes = 8192;
+constexpr int kScaleBytes = 128;
+constexpr int kZeroBytes = 32;
+constexpr int kW4TileBytes = kW4WeightBytes + kScaleBytes + kZeroBytes;   // 4256
+constexpr int kW8TileBytes = kW8WeightBytes + kScaleBytes;                // 8320
+
+}  // namespace tf

@@ -1,0 +1,151 @@
+// Host-side offline pre-tiling (Section 4.2 of the paper): AWQ / int8 weights -> packed blob.
+// Pure byte shuffling; scales are copied bit for bit.
+#include <string.h>
+
+#include "../../include/tilefuse.h"
+#include "layout.h"
+
+namespace {
+
+constexpr int kAwqPosOfColumn[8] = {0, 4, 1, 5, 2, 6, 3, 7};   // nibble position of column c%8
+
+inline uint32_t awq_code(const uint32_t* words, size_t row_words, int r, int c) {
+    return (words[(size_t)r * row_words + (c >> 3)] >> (4 * kAwqPosOfColumn[c & 7])) & 0xFu;
+}
+
+bool legal_shape(int bits, int K, int N, int g) {
+    if (bits != 4 && bits != 8) return false;
+    if (K < tf::kTileK || K > TF_MAX_DIM || N < 8 || N > TF_MAX_DIM) return false;
+    if (N % 8 != 0) return false;
+    if (g <= 0 || g % tf::kTileK != 0 || K % g != 0) return false;
+    return true;
+}
+
+void write_header(void* out, int bits, int K, int N, int g, size_t total) {
+    tf_blob_header h;
+    memset(&h, 0, sizeof(h));
+    h.magic = tf::kMagic;
+    h.version = tf::kBlobVersion;
+    h.bits = (uint32_t)bits;
+    h.K = (uint32_t)K;
+    h.N = (uint32_t)N;
+    h.group_size = (uint32_t)g;
+    h.n_padded = (uint32_t)((N + tf::kTileN - 1) / tf::kTileN * tf::kTileN);
+    h.strips = h.n_padded / tf::kTileN;
+    h.ktiles = (uint32_t)(K / tf::kTileK);
+    h.tile_bytes = bits == 4 ? tf::kW4TileBytes : tf::kW8TileBytes;
+    h.tiles_offset = tf::kHeaderBytes;
+    h.total_bytes = total;
+    memcpy(out, &h, sizeof(h));
+}
+
+// Physical (k, n) offsets inside a tile of register `reg` (0..3), element `el` (0..1) of
+// lane (g, t) in k-block kb, n-block w.
+inline void tile_coord(int kb, int g, int t, int w, int reg, int el, int* dk, int* dn) {
+    *dk = 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (reg >> 1) + el;
+    *dn = 16 * w + g + 8 * (reg & 1);
+}
+
+void write_scales(uint8_t* tile_scales, const uint16_t* scales, int N, int grp, int n0) {
+    uint16_t* s = reinterpret_cast<uint16_t*>(tile_scales);
+    for (int g = 0; g < 8; ++g)
+        for (int w = 0; w < 4; ++w)
+            for (int h = 0; h < 2; ++h) {
+                int n = n0 + 16 * w + g + 8 * h;
+                s[g * 8 + 2 * w + h] = n < N ? scales[(size_t)grp * N + n] : (uint16_t)0;
+            }
+}
+
+}  // namespace
+
+static_assert(sizeof(tf_blob_header) == tf::kHeaderBytes, "header must be 256 bytes");
+
+extern "C" __attribute__((visibility("default"))) size_t tf_packed_size(int bits, int K, int N, int group_size) {
+    if (!legal_shape(bits, K, N, group_size)) return 0;
+    size_t strips = (size_t)(N + tf::kTileN - 1) / tf::kTileN;
+    size_t ktiles = (size_t)K / tf::kTileK;
+    size_t tile = bits == 4 ? tf::kW4TileBytes : tf::kW8TileBytes;
+    return tf::kHeaderBytes + strips * ktiles * tile;
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_pack_awq(const uint32_t* qweight, const uint16_t* scales_fp16,
+                                 const uint32_t* qzeros, int K, int N, int group_size,
+                                 void* out, size_t out_bytes) {
+    if (!qweight || !scales_fp16 || !qzeros || !out) return TF_ERR_NULL;
+    size_t total = tf_packed_size(4, K, N, group_size);
+    if (total == 0) return TF_ERR_SHAPE;
+    if (out_bytes < total) return TF_ERR_WORKSPACE;
+    write_header(out, 4, K, N, group_size, total);
+    const size_t row_words = (size_t)N / 8;
+    const int strips = (N + tf::kTileN - 1) / tf::kTileN, ktiles = K / tf::kTileK;
+    uint8_t* base = static_cast<uint8_t*>(out) + tf::kHeaderBytes;
+    for (int S = 0; S < strips; ++S) {
+        const int n0 = S * tf::kTileN;
+        for (int T = 0; T < ktiles; ++T) {
+            const int k0 = T * tf::kTileK, grp = k0 / group_size;
+            uint8_t* tile = base + ((size_t)S * ktiles + T) * tf::kW4TileBytes;
+            uint32_t* wq = reinterpret_cast<uint32_t*>(tile);
+            for (int kb = 0; kb < 8; ++kb)
+                for (int lane = 0; lane < 32; ++lane)
+                    for (int w = 0; w < 4; ++w) {
+                        const int g = lane >> 2, t = lane & 3;
+                        uint32_t word = 0;
+                        for (int p = 0; p < 8; ++p) {
+                            int dk, dn;
+                            tile_coord(kb, g, t, w, p & 3, p >> 2, &dk, &dn);
+                            const int n = n0 + dn;
+                            // padded columns: q = z = 0, s = 0  ->  dequantizes to exactly 0
+                            uint32_t code = n < N ? awq_code(qweight, row_words, k0 + dk, n) : 0u;
+                            word |= code << (4 * p);
+                        }
+                        wq[(kb * 32 + lane) * 4 + w] = word;
+                    }
+            write_scales(tile + tf::kW4WeightBytes, scales_fp16, N, grp, n0);
+            uint32_t* zq = reinterpret_cast<uint32_t*>(tile + tf::kW4WeightBytes + tf::kScaleBytes);
+            for (int g = 0; g < 8; ++g) {
+                uint32_t word = 0;
+                for (int i = 0; i < 8; ++i) {
+                    const int n = n0 + 16 * (i & 3) + g + 8 * (i >> 2);
+                    uint32_t code = n < N ? awq_code(qzeros, row_words, grp, n) : 0u;
+                    word |= code << (4 * i);
+                }
+                zq[g] = word;
+            }
+        }
+    }
+    return TF_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_pack_w8(const int8_t* w8, const uint16_t* scales_fp16, int K, int N,
+                                int group_size, void* out, size_t out_bytes) {
+    if (!w8 || !scales_fp16 || !out) return TF_ERR_NULL;
+    size_t total = tf_packed_size(8, K, N, group_size);
+    if (total == 0) return TF_ERR_SHAPE;
+    if (out_bytes < total) return TF_ERR_WORKSPACE;
+    write_header(out, 8, K, N, group_size, total);
+    const int strips = (N + tf::kTileN - 1) / tf::kTileN, ktiles = K / tf::kTileK;
+    uint8_t* base = static_cast<uint8_t*>(out) + tf::kHeaderBytes;
+    for (int S = 0; S < strips; ++S) {
+        const int n0 = S * tf::kTileN;
+        for (int T = 0; T < ktiles; ++T) {
+            const int k0 = T * tf::kTileK, grp = k0 / group_size;
+            uint8_t* tile = base + ((size_t)S * ktiles + T) * tf::kW8TileBytes;
+            for (int kb = 0; kb < 8; ++kb)
+                for (int lane = 0; lane < 32; ++lane)
+                    for (int w = 0; w < 4; ++w)
+                        for (int r = 0; r < 2; ++r) {
+                            const int g = lane >> 2, t = lane & 3;
+                            uint8_t* dst = tile + (((size_t)(kb * 2 + (w >> 1)) * 32 + lane) * 4 +
+                                                   2 * (w & 1) + r) * 4;
+                            for (int b = 0; b < 4; ++b) {
+                                int dk, dn;
+                                tile_coord(kb, g, t, w, 2 * r + (b >> 1), b & 1, &dk, &dn);
+                                const int n = n0 + dn;
+                                dst[b] = n < N ? (uint8_t)w8[(size_t)(k0 + dk) * N + n] : (uint8_t)0;
+                            }
+                        }
+            write_scales(tile + tf::kW8WeightBytes, scales_fp16, N, grp, n0);
+        }
+    }
+    return TF_OK;
+}

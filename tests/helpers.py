@@ -62,3 +62,67 @@ def read_golden_dequant():
             kind, q, z, s, a, w, aw = line.split()
             cases.append((kind, int(q), int(z), float(s), float(a), float(w), float(aw)))
     return cases
+
+
+# ----------------------------------------------------------------------------------------------
+# Host-side reader of the packed blob, written from the layout description in include/tilefuse.h
+# and csrc/layout.h (test-only; the library's own decoders are the GPU kernels).
+# ----------------------------------------------------------------------------------------------
+HEADER_BYTES, TILE_K, TILE_N = 256, 128, 64
+W4_TILE, W8_TILE = 4256, 8320
+
+
+def read_header(blob):
+    h = np.frombuffer(blob[:48].tobytes(), dtype=np.uint32)
+    names = ["magic", "version", "bits", "K", "N", "group_size", "n_padded", "strips", "ktiles", "tile_bytes"]
+    out = {n: int(h[i]) for i, n in enumerate(names)}
+    tail = np.frombuffer(blob[40:56].tobytes(), dtype=np.uint64)
+    out["tiles_offset"], out["total_bytes"] = int(tail[0]), int(tail[1])
+    return out
+
+
+def read_blob(blob, bits, K, N, group_size=128):
+    """Decode a blob on the host -> (q [K, Np], z [K/128, Np] or None, s_bits [K/128, Np]) per tile row."""
+    strips, ktiles = (N + TILE_N - 1) // TILE_N, K // TILE_K
+    tile_bytes = W4_TILE if bits == 4 else W8_TILE
+    wbytes = 4096 if bits == 4 else 8192
+    tiles = blob[HEADER_BYTES:HEADER_BYTES + strips * ktiles * tile_bytes].reshape(strips, ktiles, tile_bytes)
+    Np = strips * TILE_N
+    q = np.zeros((K, Np), dtype=np.int16)
+    kb, lane, w = np.meshgrid(np.arange(8), np.arange(32), np.arange(4), indexing="ij")
+    g, t = lane >> 2, lane & 3
+    if bits == 4:
+        words = np.ascontiguousarray(tiles[:, :, :wbytes]).view(np.uint32).reshape(strips, ktiles, 8, 32, 4)
+        for p in range(8):
+            reg, el = p & 3, p >> 2
+            dk = 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (reg >> 1) + el
+            dn = 16 * w + g + 8 * (reg & 1)
+            vals = ((words >> np.uint32(4 * p)) & np.uint32(0xF)).astype(np.int16)
+            for S in range(strips):
+                for T in range(ktiles):
+                    q[T * TILE_K + dk, S * TILE_N + dn] = vals[S, T]
+    else:
+        raw = np.ascontiguousarray(tiles[:, :, :wbytes]).view(np.int8).reshape(strips, ktiles, 8, 2, 32, 4, 4)
+        for r in range(2):
+            for b in range(4):
+                reg, el = 2 * r + (b >> 1), b & 1
+                dk = 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (reg >> 1) + el
+                dn = 16 * w + g + 8 * (reg & 1)
+                for S in range(strips):
+                    for T in range(ktiles):
+                        q[T * TILE_K + dk, S * TILE_N + dn] = raw[S, T, kb, w >> 1, lane, 2 * (w & 1) + r, b]
+    sc = np.ascontiguousarray(tiles[:, :, wbytes:wbytes + 128]).view(np.uint16).reshape(strips, ktiles, 8, 4, 2)
+    s = np.zeros((ktiles, Np), dtype=np.uint16)
+    z = np.zeros((ktiles, Np), dtype=np.int16) if bits == 4 else None
+    gg, ww, hh = np.meshgrid(np.arange(8), np.arange(4), np.arange(2), indexing="ij")
+    ncol = 16 * ww + gg + 8 * hh
+    if bits == 4:
+        zw = np.ascontiguousarray(tiles[:, :, wbytes + 128:wbytes + 160]).view(np.uint32).reshape(strips, ktiles, 8)
+    for S in range(strips):
+        for T in range(ktiles):
+            s[T, S * TILE_N + ncol] = sc[S, T]
+            if bits == 4:
+                for i in range(8):
+                    z[T, S * TILE_N + 16 * (i & 3) + np.arange(8) + 8 * (i >> 2)] = \
+                        (zw[S, T] >> np.uint32(4 * i)) & np.uint32(0xF)
+    return q, z, s
