@@ -143,15 +143,19 @@ tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s_fp16,
  *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.
  *   y_bf16   device, bf16 [M][N] row-major, leading dimension N; fully overwritten.
  *   workspace, workspace_bytes   device scratch of at least tf_workspace_size(op, M, K, N)
- *            bytes (may be NULL / 0 when that size is 0).  Its first 16 bytes, when present,
- *            receive the device status word read by tf_device_status.
+ *            bytes.  Its first 4096 bytes must be zero before the first call that uses it; every
+ *            call leaves them zero again unless it reports an error there.  Bytes [0,16) hold the
+ *            device status word read by tf_device_status; the rest holds arrival counters and the
+ *            fp32 partial sums of the few column strips that are split between two CTAs.  Use one
+ *            workspace per stream: calls that run concurrently must not share one.
  * Arithmetic: weights are kept exact ((q - z) as small integers, scale applied in fp32 to
  * per-group partial sums), fp32 accumulation, one round-to-nearest-even to bf16 at the end.
- * Each CTA cluster owns a set of output columns for all K: no cross-cluster reduction.
+ * Each persistent CTA streams one contiguous range of packed tiles; a strip of 64 output
+ * columns that is cut between CTAs is summed in CTA order by the last CTA to finish it.
+ * The blob must be at least tf_packed_size(bits, K, N, 128) bytes for the K, N passed here.
  * Errors: TF_ERR_NULL, TF_ERR_SHAPE (M outside 1..16, K % 128, N % 8, limits), TF_ERR_ALIGN,
  *         TF_ERR_WORKSPACE, TF_ERR_ARCH, TF_ERR_CUDA.  A blob/argument mismatch is detected on
- *         the device: y is left untouched and the status word (if a workspace was given)
- *         becomes TF_ERR_BLOB.
+ *         the device: y is left untouched and the status word becomes TF_ERR_BLOB.
  */
 tf_status tf_gemv_w4a16(const void* packed, const void* a_bf16, void* y_bf16,
                         int M, int K, int N, void* workspace, size_t workspace_bytes,

@@ -138,12 +138,12 @@ def _linear(name, packed, a, y, M, K, N, workspace, stream):
                                       _stream(stream)))
 
 
-def tf_gemv_w4a16(packed, a, y, M, K, N, workspace=None, stream=None) -> None:
+def tf_gemv_w4a16(packed, a, y, M, K, N, workspace, stream=None) -> None:
     """a: bfloat16 [M,K], y: bfloat16 [M,N] CUDA tensors; asynchronous on the stream."""
     _linear("tf_gemv_w4a16", packed, a, y, M, K, N, workspace, stream)
 
 
-def tf_gemv_w8a16(packed, a, y, M, K, N, workspace=None, stream=None) -> None:
+def tf_gemv_w8a16(packed, a, y, M, K, N, workspace, stream=None) -> None:
     _linear("tf_gemv_w8a16", packed, a, y, M, K, N, workspace, stream)
 
 

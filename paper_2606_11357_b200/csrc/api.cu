@@ -50,12 +50,13 @@ tf_status gemv(int bits, const void* packed, const void* a, void* y, int M, int 
                size_t workspace_bytes, void* stream) {
     tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMV);
     if (st != TF_OK) return st;
-    if (workspace != nullptr && (!aligned16(workspace) || workspace_bytes < sizeof(uint32_t) * 4))
-        return workspace_bytes < 16 ? TF_ERR_WORKSPACE : TF_ERR_ALIGN;
+    if (workspace == nullptr || workspace_bytes < tf::kGemvWorkspaceBytes) return TF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return TF_ERR_ALIGN;
     DeviceInfo dev;
     st = device_info(&dev);
     if (st != TF_OK) return st;
-    const tf::GemvPlan plan = tf::plan_gemv(K, N, dev.sm_count);
+    if (dev.sm_count > tf::kGemvMaxGrid) dev.sm_count = tf::kGemvMaxGrid;
+    const tf::GemvPlan plan = tf::plan_gemv(bits, M, K, N, dev.sm_count);
     cudaError_t e = tf::launch_gemv(bits, plan, packed, a, y, M, K, N, workspace, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
     return TF_OK;
@@ -100,7 +101,8 @@ extern "C" __attribute__((visibility("default"))) size_t tf_workspace_size(int o
     const int bits = (op == TF_OP_GEMV_W4A16 || op == TF_OP_GEMM_W4A16) ? 4 : 8;
     if (op < TF_OP_GEMV_W4A16 || op > TF_OP_GEMM_W8A16) return 0;
     if (tf_packed_size(bits, K, N, tf::kTileK) == 0) return 0;
-    if (op == TF_OP_GEMV_W4A16 || op == TF_OP_GEMV_W8A16) return 0;
+    if (op == TF_OP_GEMV_W4A16 || op == TF_OP_GEMV_W8A16)
+        return (M >= 1 && M <= TF_MAX_M_GEMV) ? tf::kGemvWorkspaceBytes : 0;
     if (M < 1 || M > TF_MAX_M_GEMM) return 0;
     return tf::gemm_workspace_bytes(M, K, N);
 }

@@ -20,8 +20,18 @@ struct DeviceStatus {
 // ---- 4-bit codes -> bf16 --------------------------------------------------------------
 // bf16 0x4300 is 128.0 with a unit in the last place of 1, so OR-ing a 4-bit code into the
 // mantissa gives exactly 128 + q.  Register i of a packed word sits in nibbles i and i+4.
+// Written as one three-input logic op (a & b) | c with mask and magic held in registers; left to
+// the compiler it becomes two two-input ops because each may carry only one immediate.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
 __device__ __forceinline__ uint32_t w4_reg_biased(uint32_t word, int i) {
-    return ((word >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
+    uint32_t mask, magic;
+    asm("mov.b32 %0, 0x000F000F;" : "=r"(mask));      // opaque to constant folding on purpose
+    asm("mov.b32 %0, 0x43004300;" : "=r"(magic));
+    return and_or(word >> (4 * i), mask, magic);
 }
 
 __device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {

@@ -5,19 +5,41 @@
 
 namespace tf {
 
-constexpr int kGemvMaxThreads = 256;
+// ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
+constexpr int kGemvMaxConsumers = 12;
+constexpr int kGemvMaxThreads = 32 * (kGemvMaxConsumers + 1);
+constexpr int kGemvMaxStages = 48;
+constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
+constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
+constexpr int kGemvProducerLanes = 4;         // lanes of the producer warp that issue bulk copies
+constexpr int kGemvSmemBudget = 220 * 1024;
+// A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way).
+__host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
+__host__ __device__ constexpr int gemv_stage_bytes(int bits) {
+    return ((bits == 4 ? 4 * 4256 : 2 * 8320) + 127) / 128 * 128;
+}
+__host__ __device__ constexpr int gemv_stages(int bits, int mt) {
+    return (kGemvSmemBudget - kGemvBarrierBytes - kGemvMaxConsumers * 8 * mt * 64 * 4) / gemv_stage_bytes(bits);
+}
+constexpr int kGemvMaxM = 16;
+constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
+// Workspace layout: [0,16) status word | [256, 256+4*512) per-strip arrival counters | partial sums
+constexpr int kGemvCounterOffset = 256;
+constexpr int kGemvPartialOffset = 4096;
+constexpr size_t kGemvWorkspaceBytes = kGemvPartialOffset + (size_t)kGemvMaxGrid * 2 * kGemvMaxM * 64 * 4;
 
 struct GemvPlan {
-    int cluster;        // CTAs per cluster = K split factor (1, 2, 4 or 8)
-    int tiles_per_cta;  // k-tiles each CTA of a cluster walks
-    int threads;        // CTA size
-    int strips;         // grid.y
-    int ktiles;
+    int grid;          // persistent CTAs
+    int threads;       // 32 * (consumers + 1)
+    int consumers;     // consumer warps
+    int stages;        // ring depth
+    int smem_bytes;
+    int strips, ktiles, total_tiles;
 };
 
-GemvPlan plan_gemv(int K, int N, int sm_count);
+GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count);
 cudaError_t launch_gemv(int bits, const GemvPlan& plan, const void* blob, const void* a, void* y,
-                        int M, int K, int N, void* status, cudaStream_t stream);
+                        int M, int K, int N, void* workspace, cudaStream_t stream);
 
 cudaError_t launch_unpack_w4(const void* blob, uint8_t* q, uint8_t* z, uint16_t* s, int K, int N,
                              int group_size, cudaStream_t stream);

@@ -71,7 +71,9 @@ def test_compute_calls_validate_before_touching_the_gpu():
     assert L.tf_unpack_w4(None, ok, ok, ok, 128, 8, 128, None) == 1
     assert L.tf_unpack_w4(ok, ok, ok, ok, 128, 9, 128, None) == 2
     assert L.tf_device_status(None, None) == 1
-    assert tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 1, 4096, 4096) == 0
+    assert tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 1, 4096, 4096) >= 4096
+    assert tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 17, 4096, 4096) == 0
+    assert L.tf_gemv_w4a16(ok, ok, ok, 1, 128, 8, None, 0, None) == 5
     assert tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, 2048, 4096, 14336) >= 16
     assert tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, 5000, 4096, 14336) == 0
     assert tf.tf_workspace_size(99, 1, 4096, 4096) == 0

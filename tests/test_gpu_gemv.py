@@ -81,7 +81,7 @@ def test_mismatched_blob_reports_status_and_leaves_y():
     blob = torch.from_numpy(gu.pack(p)).cuda()
     a = gu.to_device_bf16(p.a_bf16)
     y = torch.full((1, 64), 7.0, dtype=torch.bfloat16, device="cuda")
-    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W8A16, 1, 256, 64), dtype=torch.uint8, device="cuda")
     tf.tf_gemv_w8a16(blob, a, y, 1, 256, 64, ws)                 # W4 blob handed to the W8 kernel
     assert tf.tf_device_status(ws) == 4
     assert bool((y == 7.0).all())
