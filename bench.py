@@ -1,0 +1,474 @@
+#!/usr/bin/env python
+"""Benchmark of the fused W4A16 linear layer on B200 (one process per GPU).
+
+A *step* is one decode pass over the four Llama-3-8B-shaped linear layers (K x N = 4096x4096,
+4096x1024, 4096x14336, 14336x4096) at M = 1, 4 and 16 tokens: twelve tf_gemv_w4a16 calls, each on
+its own device copy of the packed weights.  Two full sets of copies alternate between steps, so the
+weights of a call (432 MB in total) have been pushed out of the 126 MB L2 before they are read again.
+
+  value      algorithmic GB/s of the whole step, inputs resident in HBM, launches replayed from a
+             CUDA graph, timed with CUDA events on the launching stream (max over ranks).
+  e2e        the same step through the C-ABI calls one by one with HOST activations: pinned
+             host -> device copy of A and device -> host copy of Y inside the timed region.
+  gemm       the prefill GEMM (M=2048, K=4096, N=14336, 1 % outlier channels) in TFLOP/s.
+  roofline   achieved / measured-peak for the GEMV step (HBM bound); gemm.roofline likewise (tensor).
+  cpu_baseline  the fp64 CPU oracle timed on this machine's host cores on a bounded sample.
+
+`--impl reference` times the CPU oracle instead (rank 0 only).  Multi-GPU runs (`torchrun`) give
+every rank the same step on its own GPU (independent problems, no data-path collective): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+GEMV_MS = (1, 4, 16)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            data = json.load(fh)
+        return {k: float(data[k]) for k in FALLBACK_PEAKS if k in data}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic():
+    """DRAM bytes per launch from the committed ncu summaries (profiles/traffic.json), if present."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh)
+    return {}
+
+
+def gemv_algorithmic_bytes(bits, M, K, N, group=128):
+    """What the method itself must move, each byte once: weights, scales, zeros, A and Y."""
+    b = K * N * bits // 8 + (K // group) * N * 2 + M * K * 2 + M * N * 2
+    if bits == 4:
+        b += (K // group) * N // 2
+    return b
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def init_dist(backend):
+    import torch.distributed as dist
+    rank, _, world = dist_env()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29500")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, device="cpu") -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()                      # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = []
+        with open(self.path) as fh:
+            for line in fh:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) == 7:
+                    try:
+                        rows.append((float(parts[0]), float(parts[1]), float(parts[2]), parts[3:]))
+                    except ValueError:
+                        pass
+        os.unlink(self.path)
+        if not rows:
+            return out
+        busy = [r for r in rows if r[2] > 250.0] or rows          # samples under load if any
+        out["sm_mhz"] = float(np.median([r[0] for r in busy]))
+        out["sm_max_mhz"] = float(rows[0][1])
+        out["samples"] = len(busy)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for i, name in enumerate(names):
+            if any(r[3][i].lower().startswith("active") for r in busy):
+                out["reasons"].append(name)
+        return out
+
+
+# ------------------------------------------------------------------------------- CPU oracle timing
+_ORACLE_PROBLEMS = None
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return int(os.cpu_count() or 1)
+
+
+def time_oracle_sample(repeats: int = 1):
+    """The oracle as it stands on a bounded sample of the step: the four layer shapes at M = 16."""
+    from oracle import tilefuse_oracle as orc
+    from paper_2606_11357_b200 import workloads as wl
+    global _ORACLE_PROBLEMS
+    if _ORACLE_PROBLEMS is None:
+        _ORACLE_PROBLEMS = [wl.config1(16, K, N) for (K, N) in wl.LLAMA3_8B_SHAPES]
+    probs = _ORACLE_PROBLEMS
+    np.zeros(1) @ np.zeros(1)                      # make sure the BLAS threads exist before counting them
+    nbytes = sum(gemv_algorithmic_bytes(4, p.M, p.K, p.N) for p in probs)
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        for p in probs:
+            orc.solve(p)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return {"value": nbytes / best / 1e9, "unit": "GB/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": "fp64 oracle, the four Llama-3-8B layer shapes at M=16, one pass "
+                      f"({best:.2f} s, {nbytes / 1e6:.1f} MB algorithmic)"}, best, nbytes
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    for _ in range(min(args.warmup, 1)):
+        time_oracle_sample()
+    total_t, total_b = 0.0, 0
+    steps = max(1, min(args.steps, 5))             # each step is a bounded sample; keep the run to minutes
+    for _ in range(steps):
+        _, dt, nb = time_oracle_sample()
+        total_t += dt
+        total_b += nb
+    value = total_b / total_t / 1e9
+    line = {
+        "impl": "reference", "metric": "W4A16 GEMV GB/s", "value": value, "unit": "GB/s", "n_gpus": world,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": total_t / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg1 decode GEMV sweep, Llama-3-8B layer shapes (oracle sample: M=16 only)",
+                   "l2": "n/a (CPU)"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle_threads(), "kind": "oracle",
+                         "sample": "four layer shapes at M=16 per step"},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------------------- GPU bench
+def run_gpu(args):
+    import torch
+    from paper_2606_11357_b200 import binding as tf
+    from paper_2606_11357_b200 import workloads as wl
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank % torch.cuda.device_count())
+    dev = torch.device("cuda", torch.cuda.current_device())
+    init_dist("nccl")
+    tf.lib()                                        # fail loudly if the extension is missing
+    peaks, peak_kind = load_peaks()
+    traffic = load_traffic()
+
+    # ---- inputs: seeded, synthetic, resident in HBM ----------------------------------------------------
+    stream = torch.cuda.Stream()
+    ws_bytes = tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 16, 4096, 4096)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    calls = []                                       # (set, M, K, N, blob, a, y, a_host, y_host)
+    step_bytes = 0
+    for (K, N) in wl.LLAMA3_8B_SHAPES:
+        prob = wl.config1(16, K, N)
+        blob_host = tf.tf_pack_awq(prob.qweight, prob.scales_f16, prob.qzeros, K, N)
+        a_all = torch.from_numpy(prob.a_bf16.view(np.int16).copy()).view(torch.bfloat16)
+        for M in GEMV_MS:
+            step_bytes += gemv_algorithmic_bytes(4, M, K, N)
+            for s in range(2):
+                blob = torch.from_numpy(blob_host).to(dev)
+                a_host = a_all[:M].contiguous().pin_memory()
+                a = a_host.to(dev)
+                y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                y_host = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+                calls.append((s, M, K, N, blob, a, y, a_host, y_host))
+    sets = [[c for c in calls if c[0] == s] for s in range(2)]
+    launches_per_step = len(sets[0])
+
+    def enqueue_step(s):
+        for (_, M, K, N, blob, a, y, _, _) in sets[s]:
+            tf.tf_gemv_w4a16(blob, a, y, M, K, N, ws, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for s in range(2):
+            enqueue_step(s)
+    stream.synchronize()
+    if tf.tf_device_status(ws, stream=stream) != 0:
+        raise SystemExit("device status word reports an error after the first step")
+
+    # two steps (one per weight set) per graph replay
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            enqueue_step(0)
+            enqueue_step(1)
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    if rank == 0:
+        sampler.start()
+    replays_warm = max(2, (args.warmup + 1) // 2)
+    replays = max(1, (args.steps + 1) // 2)
+    steps_timed = 2 * replays
+    with torch.cuda.stream(stream):
+        for _ in range(replays_warm):
+            graph.replay()
+    stream.synchronize()
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(replays):
+            graph.replay()
+        e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    barrier()
+    ms_local = e0.elapsed_time(e1)
+    ms_total = max_over_ranks(ms_local, dev)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = ms_total / steps_timed
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host activations in, host result out, call by call ----------------------------------
+    e2e_steps = max(2, min(steps_timed, 200))
+    h2d = sum(c[7].numel() * 2 for c in sets[0])
+    d2h = sum(c[8].numel() * 2 for c in sets[0])
+
+    def e2e_step(s):
+        for (_, M, K, N, blob, a, y, a_host, y_host) in sets[s]:
+            a.copy_(a_host, non_blocking=True)
+            tf.tf_gemv_w4a16(blob, a, y, M, K, N, ws, stream=stream)
+            y_host.copy_(y, non_blocking=True)
+
+    with torch.cuda.stream(stream):
+        e2e_step(0)
+        stream.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i & 1)
+        stream.synchronize()
+        dt = time.perf_counter() - t0
+    dt = max_over_ranks(dt, dev)
+    e2e_value = world * step_bytes * e2e_steps / dt / 1e9
+
+    # ---- per-shape breakdown (graph of 2 launches on alternating copies; context for the step number) ---
+    per_shape = []
+    if rank == 0:
+        for (K, N) in wl.LLAMA3_8B_SHAPES:
+            for M in GEMV_MS:
+                pair = [c for c in calls if (c[1], c[2], c[3]) == (M, K, N)]
+                extra = []
+                nbytes = gemv_algorithmic_bytes(4, M, K, N)
+                need = int(300e6 // nbytes) + 2                      # rotate over > 2x L2 worth of copies
+                while len(pair) + len(extra) < need:
+                    extra.append(pair[0][4].clone())
+                blobs = [p[4] for p in pair] + extra
+                g = torch.cuda.CUDAGraph()
+                a, y = pair[0][5], pair[0][6]
+                with torch.cuda.stream(stream):
+                    with torch.cuda.graph(g, stream=stream):
+                        for b in blobs:
+                            tf.tf_gemv_w4a16(b, a, y, M, K, N, ws, stream=stream)
+                    g.replay()
+                    stream.synchronize()
+                    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    s0.record(stream)
+                    for _ in range(5):
+                        g.replay()
+                    s1.record(stream)
+                    stream.synchronize()
+                us = s0.elapsed_time(s1) * 1e3 / (5 * len(blobs))
+                per_shape.append({"M": M, "K": K, "N": N, "us": round(us, 3), "GBps": round(nbytes / us / 1e3, 1),
+                                  "frac_of_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
+                del g, extra, blobs
+
+    # ---- prefill GEMM (config 2) ---------------------------------------------------------------------------
+    gemm = None
+    if rank == 0 and not args.skip_gemm:
+        p2 = wl.config2()
+        blob = torch.from_numpy(tf.tf_pack_awq(p2.qweight, p2.scales_f16, p2.qzeros, p2.K, p2.N)).to(dev)
+        a = torch.from_numpy(p2.a_bf16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+        y = torch.empty((p2.M, p2.N), dtype=torch.bfloat16, device=dev)
+        gws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, p2.M, p2.K, p2.N), dtype=torch.uint8, device=dev)
+        iters = 20
+        with torch.cuda.stream(stream):
+            for _ in range(5):
+                tf.tf_gemm_w4a16(blob, a, y, p2.M, p2.K, p2.N, gws, stream=stream)
+            stream.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+            for _ in range(iters):
+                tf.tf_gemm_w4a16(blob, a, y, p2.M, p2.K, p2.N, gws, stream=stream)
+            g1.record(stream)
+            stream.synchronize()
+        if tf.tf_device_status(gws, stream=stream) != 0:
+            raise SystemExit("GEMM device status word reports an error")
+        us = g0.elapsed_time(g1) * 1e3 / iters
+        flops = 2.0 * p2.M * p2.K * p2.N
+        tfl = flops / us / 1e6
+        gemm = {"metric": "W4A16 GEMM TFLOP/s", "value": tfl, "unit": "TFLOP/s", "us_per_launch": us,
+                "workload": f"cfg2 prefill GEMM M={p2.M} K={p2.K} N={p2.N}, 1% outlier channels x20",
+                "dtype": "bf16", "gpu_launches": iters,
+                "roofline": {"bound": "tensor", "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                             "frac": tfl / peaks["bf16_tflops"], "peak_kind": f"{peak_kind} (burst, cuBLAS bf16)",
+                             "traffic": traffic.get("gemm_w4_cfg2_dram_bytes_per_launch")}}
+
+    if rank != 0:
+        return 0
+    cpu_baseline = None
+    if not args.skip_cpu:
+        cpu_baseline, _, _ = time_oracle_sample()
+    achieved = step_bytes / (ms_local / steps_timed * 1e-3) / 1e9
+    line = {
+        "metric": "W4A16 GEMV GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps_timed,
+        "warmup": 2 * replays_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg1 decode GEMV sweep: Llama-3-8B layer shapes 4096x4096, 4096x1024, 4096x14336, "
+                               "14336x4096 at M=1,4,16 (12 tf_gemv_w4a16 calls per step)",
+                   "l2": "inputs larger than L2: two alternating sets of 12 weight copies, 432 MB in rotation",
+                   "bytes_per_step": step_bytes, "launch": "CUDA graph replay of two steps"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": launches_per_step * steps_timed,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"{peak_kind} (copy bandwidth)",
+                     "traffic": traffic.get("gemv_w4_step_dram_bytes"),
+                     "kernel": "gemv_stream_kernel (all 12 launches of the step)"},
+        "cpu_baseline": cpu_baseline,
+        "per_shape": per_shape,
+        "gemm": gemm,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def run_profile_case(args):
+    """A handful of launches of one kernel on one seeded case, for `ncu` captures (prints no bench line)."""
+    import torch
+    from paper_2606_11357_b200 import binding as tf
+    from paper_2606_11357_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    kind, bits = args.profile_case.split("_")
+    bits = int(bits[1])
+    if kind == "gemv":
+        prob = (wl.config1(args.profile_m or 1, 4096, 14336) if bits == 4 else wl.config3_gemv())
+    else:
+        prob = (wl.config2(args.profile_m or 2048) if bits == 4 else wl.config3_gemm())
+    M, K, N = prob.M, prob.K, prob.N
+    host = (tf.tf_pack_awq(prob.qweight, prob.scales_f16, prob.qzeros, K, N) if bits == 4
+            else tf.tf_pack_w8(prob.w_i8, prob.scales_f16, K, N))
+    copies = [torch.from_numpy(host).cuda() for _ in range(max(1, args.steps))]
+    a = torch.from_numpy(prob.a_bf16.view(np.int16).copy()).cuda().view(torch.bfloat16)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    op = {("gemv", 4): 0, ("gemv", 8): 1, ("gemm", 4): 2, ("gemm", 8): 3}[(kind, bits)]
+    ws = torch.zeros(tf.tf_workspace_size(op, M, K, N), dtype=torch.uint8, device="cuda")
+    fn = getattr(tf, f"tf_{kind}_w{bits}a16")
+    for blob in copies:
+        fn(blob, a, y, M, K, N, ws)
+    torch.cuda.synchronize()
+    status = tf.tf_device_status(ws)
+    print(json.dumps({"profile_case": args.profile_case, "M": M, "K": K, "N": N, "launches": len(copies),
+                      "device_status": status}), flush=True)
+    return 0 if status == 0 else 1
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--skip-gemm", action="store_true", help="leave out the prefill GEMM section")
+    ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline")
+    ap.add_argument("--profile-case", choices=["gemv_w4", "gemv_w8", "gemm_w4", "gemm_w8"], default=None,
+                    help="run --steps launches of one kernel on one case and exit (for ncu captures)")
+    ap.add_argument("--profile-m", type=int, default=0, help="token count for --profile-case")
+    args = ap.parse_args(argv)
+    if args.profile_case:
+        return run_profile_case(args)
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
