@@ -4,16 +4,23 @@
 // weights are the 128-row operand of the tensor-core instruction, the activations the BT-column one,
 //     D[n, token] = sum_k W[n, k] * A[token, k]          (tcgen05.mma, bf16 x bf16 -> fp32 in TMEM)
 // so that each packed weight is unpacked and dequantized exactly once per CTA tile and then reused by
-// all BT token rows (the dequantize-once rule of Section 4.1) and the dequant cost is as small as it
-// can be relative to the MMA work.
+// all BT token rows (the dequantize-once rule of Section 4.1).
+//
+// The dequantized weights never touch shared memory: the dequant warps write them with tcgen05.st
+// straight into tensor memory, from where tcgen05.mma reads its 128-row operand.  Shared memory then
+// carries only the packed 4/8-bit tiles and the activations, which is what keeps the tensor pipe fed:
+// with the bf16 weights staged in shared memory the kernel was bound by shared-memory bandwidth.
+// Tensor memory (512 columns): accumulator [0, BT), weight-operand ring [256, 256 + 4 x 32).
 //
 // Persistent, warp-specialised CTA (512 threads):
-//   warp 0      producer: bulk (TMA) copies of packed weight tiles (payload = weights + their scales
-//               and zeros, Section 4.2) and tiled TMA loads of the activation tile (128B swizzle).
-//   warp 1      one thread issues tcgen05.mma (4 per 64-wide k-step) and tcgen05.commit.
-//   warp 2      allocates / frees tensor memory (two accumulators: epilogue overlaps the next tile).
-//   warps 4-11  dequantize: packed words -> (q - z) exact in bf16 -> times bf16 scale -> bf16 operand
-//               in shared memory in the K-major 128B-swizzled layout the MMA reads.
+//   warp 0      producer A: tiled TMA loads of the activation tile (128B swizzle), one per 64-wide k-step.
+//   warp 3      producer W: bulk (TMA) copies of packed weight tiles (payload = weights + their scales
+//               and zeros, Section 4.2).
+//   warp 1      one thread issues tcgen05.mma (4 per k-step) and tcgen05.commit.
+//   warp 2      allocates / frees tensor memory.
+//   warps 4-11  dequantize: packed words -> (q - z) exact in bf16 -> times bf16 scale -> tcgen05.st.  The
+//               packed words are stored in the register order of the 16x256b store, so a word goes from
+//               shared memory to the tensor-memory operand without any shuffle.
 //   warps 12-15 epilogue: tcgen05.ld accumulator -> bf16 -> y.
 // Every mbarrier wait is bounded; on a timeout all roles leave, TMEM is freed, the status word is set.
 #include <cuda.h>
@@ -28,28 +35,36 @@ namespace {
 
 constexpr int kGemmThreads = 512;
 constexpr int kBN = 128;                  // weight columns per CTA tile (two packed strips)
-constexpr int kBK = 64;                   // k per pipeline step (one 128-byte swizzled row)
-constexpr int kStages = 4;                // activation / dequantized-weight ring depth
-constexpr int kAStageBytes = kBN * kBK * 2;            // 16 KB of dequantized weights per k-step
-constexpr int kMaxWpStages = 3;
+constexpr int kBK = 64;                   // k per pipeline step (one 128-byte swizzled activation row)
+constexpr int kAStages = 4;               // weight-operand ring in tensor memory (32 columns per k-step)
+constexpr int kTmemAccCols = 256;
+constexpr int kTmemCols = 512;
+constexpr int kMaxActStages = 12;
+constexpr int kWpStages = 3;              // packed-weight ring (one stage = the two strip tiles of one k-tile)
 
-// packed-weight ring: one stage = the two strip tiles of one k-tile (= two k-steps)
 __host__ __device__ constexpr int wp_strip_bytes(int bits) { return bits == 4 ? 4352 : 8320; }
-__host__ __device__ constexpr int wp_stages(int bits) { return bits == 4 ? 3 : 2; }
 __host__ __device__ constexpr int act_stage_bytes(int bt) { return bt * kBK * 2; }
+// activation ring depth: as deep as fits beside the packed ring, at most kMaxActStages
+__host__ __device__ constexpr int act_stages(int bits, int bt) {
+    return (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt) > kMaxActStages
+               ? kMaxActStages
+               : (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt);
+}
+constexpr int kEpiWarpBytes = 1024;       // per epilogue warp: 16 tokens x 32 columns of bf16, for the transpose
 __host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
-    return 1024 /*alignment slack*/ + kStages * (act_stage_bytes(bt) + kAStageBytes) +
-           wp_stages(bits) * 2 * wp_strip_bytes(bits) + 1024;
+    return 1024 /*alignment slack*/ + act_stages(bits, bt) * act_stage_bytes(bt) +
+           kWpStages * 2 * wp_strip_bytes(bits) + 4 * kEpiWarpBytes + 512;
 }
 
 struct GemmBarriers {
-    uint64_t act_full[kStages];
-    uint64_t w_full[kStages];
-    uint64_t ab_empty[kStages];
-    uint64_t wp_full[kMaxWpStages];
-    uint64_t wp_empty[kMaxWpStages];
-    uint64_t acc_full[2];
-    uint64_t acc_empty[2];
+    uint64_t act_full[kMaxActStages];
+    uint64_t act_empty[kMaxActStages];
+    uint64_t a_full[kAStages];
+    uint64_t a_empty[kAStages];
+    uint64_t wp_full[kWpStages];
+    uint64_t wp_empty[kWpStages];
+    uint64_t acc_full;
+    uint64_t acc_empty;
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -69,18 +84,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kActStage = act_stage_bytes(BT);
-    constexpr int kWpStages = wp_stages(BITS);
+    constexpr int kStages = act_stages(BITS, BT);
     constexpr int kWpStripBytes = wp_strip_bytes(BITS);
     constexpr int kWpStageBytes = 2 * kWpStripBytes;
-    constexpr uint32_t kTmemCols = 2 * BT < 32 ? 32 : 2 * BT;
     constexpr uint32_t kIdesc = umma_idesc_bf16(kBN, BT);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* act_ring = smem;                                        // kStages x kActStage   (1024-aligned)
-    uint8_t* a_ring = act_ring + kStages * kActStage;                // kStages x 16 KB        (1024-aligned)
-    uint8_t* wp_ring = a_ring + kStages * kAStageBytes;              // kWpStages x packed tiles
-    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(wp_ring + kWpStages * kWpStageBytes);
+    uint8_t* wp_ring = act_ring + kStages * kActStage;               // kWpStages x packed tiles
+    uint8_t* epi_buf = wp_ring + kWpStages * kWpStageBytes;          // 4 x kEpiWarpBytes
+    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(epi_buf + 4 * kEpiWarpBytes);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -92,17 +106,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&bars->act_full[s]), 1);
-            mbar_init(smem_u32(&bars->w_full[s]), 4);        // the four dequant warps of one k-half
-            mbar_init(smem_u32(&bars->ab_empty[s]), 1);      // tcgen05.commit
+            mbar_init(smem_u32(&bars->act_empty[s]), 1);     // tcgen05.commit
+        }
+        for (int s = 0; s < kAStages; ++s) {
+            mbar_init(smem_u32(&bars->a_full[s]), 4);        // the four dequant warps (lane quarters) of one k-half
+            mbar_init(smem_u32(&bars->a_empty[s]), 1);       // tcgen05.commit
         }
         for (int s = 0; s < kWpStages; ++s) {
             mbar_init(smem_u32(&bars->wp_full[s]), 1);
             mbar_init(smem_u32(&bars->wp_empty[s]), 8);      // all eight dequant warps
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&bars->acc_full[b]), 1);
-            mbar_init(smem_u32(&bars->acc_empty[b]), 4);     // four epilogue warps
-        }
+        mbar_init(smem_u32(&bars->acc_full), 1);
+        mbar_init(smem_u32(&bars->acc_empty), 4);            // four epilogue warps
         bars->abort_flag = 0;
         mbar_init_fence();
     }
@@ -114,18 +129,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
+    const uint32_t tmem_a = tmem_base + kTmemAccCols;        // weight-operand ring
 
     if (header_ok) {
         if (warp == 0 && lane == 0) {
-            // ================= producer ====================================================================
+            // ================= producer A: activation tile, one TMA load per k-step ==========================
             prefetch_tensormap(&act_map);
-            uint32_t it = 0, wit = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
+                for (int ks = 0; ks < 2 * ktiles; ++ks, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(smem_u32(&bars->act_empty[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x310 + s);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars->act_full[s]), kActStage);
+                    tma_load_2d(smem_u32(act_ring + s * kActStage), &act_map, ks * kBK, m_tile * BT,
+                                smem_u32(&bars->act_full[s]));
+                }
+            }
+        } else if (warp == 3 && lane == 0) {
+            // ================= producer W: packed weight tiles (weights + scales + zeros in one payload) =====
+            uint32_t wit = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int n_tile = tile / m_tiles;
                 const int strip0 = 2 * n_tile;
                 const int nstrips = (strip0 + 1 < strips) ? 2 : 1;
-                bool ok = true;
-                for (int T = 0; T < ktiles && ok; ++T, ++wit) {
+                for (int T = 0; T < ktiles; ++T, ++wit) {
                     const int ws = wit % kWpStages;
                     ok = mbar_wait(smem_u32(&bars->wp_empty[ws]), ((wit / kWpStages) & 1) ^ 1, abort_flag, 0x300 + ws);
                     if (!ok) break;
@@ -134,50 +165,40 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                         bulk_copy_g2s(smem_u32(wp_ring + ws * kWpStageBytes + q * kWpStripBytes),
                                       blob + kHeaderBytes + ((size_t)(strip0 + q) * ktiles + T) * kTileBytes, kTileBytes,
                                       smem_u32(&bars->wp_full[ws]));
-                    for (int half = 0; half < 2; ++half, ++it) {
-                        const int s = it % kStages;
-                        ok = mbar_wait(smem_u32(&bars->ab_empty[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x310 + s);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(smem_u32(&bars->act_full[s]), kActStage);
-                        tma_load_2d(smem_u32(act_ring + s * kActStage), &act_map, T * kTileK + half * kBK, m_tile * BT,
-                                    smem_u32(&bars->act_full[s]));
-                    }
                 }
-                if (!ok) break;
             }
         } else if (warp == 1 && lane == 0) {
             // ================= MMA issuer ==================================================================
             uint32_t it = 0, tile_it = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
-                const int buf = tile_it & 1;
-                if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), ((tile_it >> 1) & 1) ^ 1, abort_flag, 0x400 + buf)) break;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+                ok = mbar_wait(smem_u32(&bars->acc_empty), (tile_it & 1) ^ 1, abort_flag, 0x400);
+                if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BT;
-                bool ok = true;
                 for (int ks = 0; ks < 2 * ktiles; ++ks, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
-                    ok = mbar_wait(smem_u32(&bars->w_full[s]), ph, abort_flag, 0x410 + s) &&
-                         mbar_wait(smem_u32(&bars->act_full[s]), ph, abort_flag, 0x420 + s);
+                    const int s = it % kStages, sa = it % kAStages;
+                    ok = mbar_wait(smem_u32(&bars->a_full[sa]), (it / kAStages) & 1, abort_flag, 0x410 + sa) &&
+                         mbar_wait(smem_u32(&bars->act_full[s]), (it / kStages) & 1, abort_flag, 0x420 + s);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t a_desc = umma_desc_k_sw128(smem_u32(a_ring + s * kAStageBytes));
                     const uint64_t b_desc = umma_desc_k_sw128(smem_u32(act_ring + s * kActStage));
 #pragma unroll
-                    for (int j = 0; j < kBK / 16; ++j)       // 16 k per instruction = 32 bytes along the swizzled row
-                        tc_mma_f16(d_tmem, a_desc + 2 * j, b_desc + 2 * j, kIdesc, (ks | j) != 0 ? 1u : 0u);
-                    tc_commit(smem_u32(&bars->ab_empty[s]));
+                    for (int j = 0; j < kBK / 16; ++j)       // 16 k per instruction: 8 TMEM columns / 32 smem bytes
+                        tc_mma_f16_tmem_a(tmem_base, tmem_a + 32 * sa + 8 * j, b_desc + 2 * j, kIdesc, (ks | j) != 0 ? 1u : 0u);
+                    tc_commit(smem_u32(&bars->act_empty[s]));
+                    tc_commit(smem_u32(&bars->a_empty[sa]));
                 }
                 if (!ok) break;
-                tc_commit(smem_u32(&bars->acc_full[buf]));
+                tc_commit(smem_u32(&bars->acc_full));
             }
         } else if (warp >= 4 && warp < 12) {
-            // ================= dequantize: packed tile -> bf16 MMA operand ===================================
-            const int dw = warp - 4;
-            const int half = dw >> 2, strip_sel = (dw >> 1) & 1, kpl = dw & 1;
-            const int kp = 2 * half + kpl;                   // k-block pair (kb = 2kp, 2kp+1) of the 128-k tile
-            const int g = lane >> 2, t = lane & 3;
-            const int chunk = 2 * t + kpl;                   // 16-byte chunk of the 128-byte row: k = 8*chunk .. +7
+            // ================= dequantize: packed tile -> bf16 operand in tensor memory ========================
+            // warp -> (TMEM lane quarter q = 32 weight columns, k-half of the tile).  Quarter q covers strip q>>1,
+            // 16-column blocks w0 = 2(q&1) and w0+1.  Thread (g, t) owns rows g, g+8 of both blocks and, per
+            // k-block, the four consecutive k its packed word holds.
+            const int q = warp & 3, half = (warp - 4) >> 2;
+            const int strip_sel = q >> 1, w0 = 2 * (q & 1);
+            const int g = lane >> 2;
             uint32_t wit = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -188,103 +209,108 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     ok = mbar_wait(smem_u32(&bars->wp_full[ws]), (wit / kWpStages) & 1, abort_flag, 0x500 + ws);
                     if (!ok) break;
                     const uint8_t* tile_smem = wp_ring + ws * kWpStageBytes + strip_sel * kWpStripBytes;
-                    // operands of this thread: rows 16w+g and 16w+g+8 (w = 0..3), 8 consecutive k
-                    uint32_t lo_g[4][2], lo_g8[4][2], hi_g[4][2], hi_g8[4][2];   // [w][k-pair] for k 0..3 / 4..7
-                    const uint4 sc = *(reinterpret_cast<const uint4*>(tile_smem + kWeightBytes) + g);
-                    if (BITS == 4) {
-                        const uint4 x0 = *reinterpret_cast<const uint4*>(tile_smem + ((2 * kp) * 32 + lane) * 16);
-                        const uint4 x1 = *reinterpret_cast<const uint4*>(tile_smem + ((2 * kp + 1) * 32 + lane) * 16);
-                        const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile_smem + kWeightBytes + kScaleBytes) + g);
-                        uint32_t zg[4], zg8[4];
-                        w4_zero_regs(zword, zg, zg8);
-                        const uint32_t xs0[4] = {x0.x, x0.y, x0.z, x0.w}, xs1[4] = {x1.x, x1.y, x1.z, x1.w};
+                    uint32_t op[2][16];                        // [block][register of the 16x256b.x4 store]
+                    // scales of rows (w0,g), (w0,g+8), (w0+1,g), (w0+1,g+8)
+                    const uint2 sc = *(reinterpret_cast<const uint2*>(tile_smem + kWeightBytes + g * 16) + (q & 1));
+                    const uint32_t sw[2] = {sc.x, sc.y};
+                    uint32_t s_g[2], s_g8[2];
 #pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            lo_g[w][0] = bf16x2_sub(w4_reg_biased(xs0[w], 0), zg[w]);
-                            lo_g8[w][0] = bf16x2_sub(w4_reg_biased(xs0[w], 1), zg8[w]);
-                            lo_g[w][1] = bf16x2_sub(w4_reg_biased(xs0[w], 2), zg[w]);
-                            lo_g8[w][1] = bf16x2_sub(w4_reg_biased(xs0[w], 3), zg8[w]);
-                            hi_g[w][0] = bf16x2_sub(w4_reg_biased(xs1[w], 0), zg[w]);
-                            hi_g8[w][0] = bf16x2_sub(w4_reg_biased(xs1[w], 1), zg8[w]);
-                            hi_g[w][1] = bf16x2_sub(w4_reg_biased(xs1[w], 2), zg[w]);
-                            hi_g8[w][1] = bf16x2_sub(w4_reg_biased(xs1[w], 3), zg8[w]);
+                    for (int b = 0; b < 2; ++b) {
+                        s_g[b] = bf16_dup(fp16_bits_to_float((uint16_t)(sw[b] & 0xFFFFu)));
+                        s_g8[b] = bf16_dup(fp16_bits_to_float((uint16_t)(sw[b] >> 16)));
+                    }
+                    if (BITS == 4) {
+                        const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile_smem + kWeightBytes + kScaleBytes) + g);
+                        uint32_t zg[2], zg8[2];
+#pragma unroll
+                        for (int b = 0; b < 2; ++b) {
+                            const uint32_t pair = w4_reg_biased(zword, w0 + b);   // (128 + z[row g], 128 + z[row g+8])
+                            zg[b] = __byte_perm(pair, 0, 0x1010);
+                            zg8[b] = __byte_perm(pair, 0, 0x3232);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {              // k-block 4*half + i = MMA k-step i of this operand stage
+                            const uint2 x = *(reinterpret_cast<const uint2*>(tile_smem + ((4 * half + i) * 32 + lane) * 16) + (q & 1));
+                            const uint32_t xs[2] = {x.x, x.y};
+#pragma unroll
+                            for (int b = 0; b < 2; ++b) {
+                                op[b][4 * i + 0] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 0), zg[b]), s_g[b]);    // row g,   k 0,1
+                                op[b][4 * i + 1] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 2), zg[b]), s_g[b]);    // row g,   k 2,3
+                                op[b][4 * i + 2] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 1), zg8[b]), s_g8[b]);  // row g+8, k 0,1
+                                op[b][4 * i + 3] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 3), zg8[b]), s_g8[b]);  // row g+8, k 2,3
+                            }
                         }
                     } else {
 #pragma unroll
-                        for (int h2 = 0; h2 < 2; ++h2) {
-                            const uint4 x0 = *reinterpret_cast<const uint4*>(tile_smem + (((2 * kp) * 2 + h2) * 32 + lane) * 16);
-                            const uint4 x1 = *reinterpret_cast<const uint4*>(tile_smem + (((2 * kp + 1) * 2 + h2) * 32 + lane) * 16);
-                            w8_word_to_regs(x0.x, lo_g[2 * h2][0], lo_g8[2 * h2][0]);
-                            w8_word_to_regs(x0.y, lo_g[2 * h2][1], lo_g8[2 * h2][1]);
-                            w8_word_to_regs(x0.z, lo_g[2 * h2 + 1][0], lo_g8[2 * h2 + 1][0]);
-                            w8_word_to_regs(x0.w, lo_g[2 * h2 + 1][1], lo_g8[2 * h2 + 1][1]);
-                            w8_word_to_regs(x1.x, hi_g[2 * h2][0], hi_g8[2 * h2][0]);
-                            w8_word_to_regs(x1.y, hi_g[2 * h2][1], hi_g8[2 * h2][1]);
-                            w8_word_to_regs(x1.z, hi_g[2 * h2 + 1][0], hi_g8[2 * h2 + 1][0]);
-                            w8_word_to_regs(x1.w, hi_g[2 * h2 + 1][1], hi_g8[2 * h2 + 1][1]);
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 x = *reinterpret_cast<const uint4*>(tile_smem + (((4 * half + i) * 2 + (q & 1)) * 32 + lane) * 16);
+                            const uint32_t xs[2][2] = {{x.x, x.y}, {x.z, x.w}};
+#pragma unroll
+                            for (int b = 0; b < 2; ++b) {
+                                uint32_t r0, r1, r2, r3;
+                                w8_word_to_regs(xs[b][0], r0, r1);                     // (row g; k 0,1), (row g+8; k 0,1)
+                                w8_word_to_regs(xs[b][1], r2, r3);                     // (row g; k 2,3), (row g+8; k 2,3)
+                                op[b][4 * i + 0] = bf16x2_mul(r0, s_g[b]);
+                                op[b][4 * i + 1] = bf16x2_mul(r2, s_g[b]);
+                                op[b][4 * i + 2] = bf16x2_mul(r1, s_g8[b]);
+                                op[b][4 * i + 3] = bf16x2_mul(r3, s_g8[b]);
+                            }
                         }
                     }
-                    // the packed stage is in registers now
+                    // the packed stage has been read
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars->wp_empty[ws]));
 
-                    // wait until the MMAs that read this operand stage (kStages steps ago) are done
+                    // wait until the MMAs that read this operand stage (kAStages steps ago) are done
                     const uint32_t it = 2 * wit + half;
-                    const int s = it % kStages;
-                    ok = mbar_wait(smem_u32(&bars->ab_empty[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x510 + s);
+                    const int sa = it % kAStages;
+                    ok = mbar_wait(smem_u32(&bars->a_empty[sa]), ((it / kAStages) & 1) ^ 1, abort_flag, 0x510 + sa);
                     if (!ok) break;
-                    uint8_t* a_stage = a_ring + s * kAStageBytes;
+                    tc_fence_after();
                     if (strip_exists) {
-                        const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            const uint32_t s_g = bf16_dup(fp16_bits_to_float((uint16_t)(sw[w] & 0xFFFFu)));
-                            const uint32_t s_g8 = bf16_dup(fp16_bits_to_float((uint16_t)(sw[w] >> 16)));
-                            const int row = 64 * strip_sel + 16 * w + g;                  // row & 7 == g
-                            uint4 v;
-                            v.x = bf16x2_mul(lo_g[w][0], s_g);
-                            v.y = bf16x2_mul(lo_g[w][1], s_g);
-                            v.z = bf16x2_mul(hi_g[w][0], s_g);
-                            v.w = bf16x2_mul(hi_g[w][1], s_g);
-                            *reinterpret_cast<uint4*>(a_stage + row * 128 + ((chunk ^ g) << 4)) = v;
-                            v.x = bf16x2_mul(lo_g8[w][0], s_g8);
-                            v.y = bf16x2_mul(lo_g8[w][1], s_g8);
-                            v.z = bf16x2_mul(hi_g8[w][0], s_g8);
-                            v.w = bf16x2_mul(hi_g8[w][1], s_g8);
-                            *reinterpret_cast<uint4*>(a_stage + (row + 8) * 128 + ((chunk ^ g) << 4)) = v;
-                        }
+                        const uint32_t taddr = tmem_a + 32 * sa + (uint32_t(32 * q) << 16);
+                        tmem_st_16x256b_x4(taddr, op[0]);
+                        tmem_st_16x256b_x4(taddr + (16u << 16), op[1]);
+                        tmem_st_wait();
                     }
-                    fence_proxy_async_smem();                 // generic-proxy stores -> visible to the MMA
+                    tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars->w_full[s]));
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[sa]));
                 }
             }
         } else if (warp >= 12) {
             // ================= epilogue: TMEM -> bf16 -> y ===================================================
-            const int quarter = warp - 12;                    // this warp may touch TMEM lanes 32*quarter .. +31
+            const int quarter = warp & 3;                     // this warp may touch TMEM lanes 32*quarter .. +31
             uint32_t tile_it = 0;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
                 const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
-                const int buf = tile_it & 1;
-                if (!mbar_wait(smem_u32(&bars->acc_full[buf]), (tile_it >> 1) & 1, abort_flag, 0x600 + buf)) break;
+                if (!mbar_wait(smem_u32(&bars->acc_full), tile_it & 1, abort_flag, 0x600)) break;
                 tc_fence_after();
-                const int n = n_tile * kBN + 32 * quarter + lane;
-                const uint32_t taddr = tmem_base + (uint32_t(32 * quarter) << 16) + buf * BT;
+                // A thread reads 16 tokens of its own column n from TMEM; the warp transposes them through a
+                // private 1 KB buffer so that each thread then stores 8 consecutive columns (16 bytes) of one token.
+                const uint32_t taddr = tmem_base + (uint32_t(32 * quarter) << 16);
+                __nv_bfloat16* tbuf = reinterpret_cast<__nv_bfloat16*>(epi_buf + quarter * kEpiWarpBytes);   // [16][32]
+                const int n8 = n_tile * kBN + 32 * quarter + 8 * (lane & 3);     // first of this thread's 8 columns
 #pragma unroll 1
-                for (int c = 0; c < BT / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld_32x32b_x32(taddr + 32 * c, v);
+                for (int c = 0; c < BT / 16; ++c) {
+                    uint32_t v[16];
+                    tmem_ld_32x32b_x16(taddr + 16 * c, v);
                     tmem_ld_wait();
-                    const int tok0 = m_tile * BT + 32 * c;
-                    if (n < N) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (tok0 + j < M) y[(size_t)(tok0 + j) * N + n] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    for (int j = 0; j < 16; ++j) tbuf[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const int tl = 8 * i + (lane >> 2);
+                        const int tok = m_tile * BT + 16 * c + tl;
+                        const uint4 d = *reinterpret_cast<const uint4*>(tbuf + tl * 32 + 8 * (lane & 3));
+                        if (tok < M && n8 < N) *reinterpret_cast<uint4*>(y + (size_t)tok * N + n8) = d;
                     }
+                    __syncwarp();
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty));
             }
         }
     }

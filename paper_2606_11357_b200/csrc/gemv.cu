@@ -123,22 +123,14 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             int j = i + ((cw - (i % nconsumers)) + nconsumers) % nconsumers;
             for (; j < i + seg_len; j += nconsumers) {
                 const int T = T0 + (j - i);
-                // activations of this k-tile: lane (g, t) holds token g (+8), k = 64c + 16t .. +15
-                uint4 av[MT][2][2];
+                // activations of this k-tile: lane (g, t) holds token g (+8), k = 16kb + 4t .. +3 per k-block
+                uint2 av[MT][8];
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     const int m = g + 8 * mt;
+                    const uint2* ap = reinterpret_cast<const uint2*>(a + (size_t)(m < M ? m : 0) * K + T * kTileK + 4 * t);
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        if (m < M) {
-                            const uint4* ap = reinterpret_cast<const uint4*>(a + (size_t)m * K + T * kTileK + 64 * c + 16 * t);
-                            av[mt][c][0] = __ldg(ap);
-                            av[mt][c][1] = __ldg(ap + 1);
-                        } else {
-                            av[mt][c][0] = make_uint4(0, 0, 0, 0);
-                            av[mt][c][1] = make_uint4(0, 0, 0, 0);
-                        }
-                    }
+                    for (int kb = 0; kb < 8; ++kb) av[mt][kb] = m < M ? __ldg(ap + 4 * kb) : make_uint2(0u, 0u);
                 }
                 const int chunk = j / kR;
                 const int s = chunk % nstages;
@@ -164,9 +156,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     uint32_t b0[MT], b1[MT];
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        const uint4 v = av[mt][kb >> 2][(kb & 3) >> 1];
-                        b0[mt] = (kb & 1) ? v.z : v.x;
-                        b1[mt] = (kb & 1) ? v.w : v.y;
+                        b0[mt] = av[mt][kb].x;
+                        b1[mt] = av[mt][kb].y;
                     }
                     uint4 wv[kVecPerKb];
 #pragma unroll

@@ -3,13 +3,15 @@
 // A tile covers TF_TILE_K = 128 rows (k) x TF_TILE_N = 64 columns (n).  Its weights are stored
 // in the register order of the warp-level tensor-core operand "A" of shape 16 (n) x 16 (k):
 // lane L = (g << 2) | t  (g = 0..7, t = 0..3) owns, per 16x16 block, four bf16x2 registers
-//     r0 = (row g,   k-slots 2t,2t+1)      r1 = (row g+8, k-slots 2t,2t+1)
-//     r2 = (row g,   k-slots 2t+8,2t+9)    r3 = (row g+8, k-slots 2t+8,2t+9)
-// A tile has 8 k-blocks (kb) x 4 n-blocks (w).  The contraction index may be permuted freely as
-// long as weights and activations agree, so k-slots map to physical k such that one lane reads
-// 16 consecutive activations for four consecutive k-blocks:
-//     k = k0 + 64*(kb>>2) + 16*t + 4*(kb&3) + {0,1 (r0/r1 lo,hi), 2,3 (r2/r3 lo,hi)}
+//     r0 = (row g,   k 4t, 4t+1)      r1 = (row g+8, k 4t, 4t+1)
+//     r2 = (row g,   k 4t+2, 4t+3)    r3 = (row g+8, k 4t+2, 4t+3)
+// A tile has 8 k-blocks (kb, 16 k each) x 4 n-blocks (w, 16 n each):
+//     k = k0 + 16*kb + 4*t + {0,1 (r0/r1 lo,hi), 2,3 (r2/r3 lo,hi)}
 //     n = n0 + 16*w + g + 8*(register is r1 or r3)
+// (The warp-level MMA numbers its k-slots 2t,2t+1,2t+8,2t+9; the contraction index may be permuted
+// freely as long as weights and activations agree, and this choice gives every lane four consecutive
+// k -- one 8-byte activation load -- and is also the register order of the 16x256b tensor-memory
+// store, so the GEMM can move a word straight into the TMEM operand of tcgen05.mma.)
 //
 // W4: one uint32 per (kb, lane, w) at word index (kb*32 + lane)*4 + w; nibble p holds register
 //     (p & 3), element (p >> 2)  -- so  (x >> 4*i) & 0x000F000F  is register i as two integers.

@@ -42,7 +42,7 @@ void write_header(void* out, int bits, int K, int N, int g, size_t total) {
 // Physical (k, n) offsets inside a tile of register `reg` (0..3), element `el` (0..1) of
 // lane (g, t) in k-block kb, n-block w.
 inline void tile_coord(int kb, int g, int t, int w, int reg, int el, int* dk, int* dn) {
-    *dk = 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (reg >> 1) + el;
+    *dk = 16 * kb + 4 * t + 2 * (reg >> 1) + el;
     *dn = 16 * w + g + 8 * (reg & 1);
 }
 

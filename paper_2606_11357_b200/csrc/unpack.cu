@@ -42,7 +42,7 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ blob, uint8_t* __restr
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int el = 0; el < 2; ++el) {
-                const int k = k0 + 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (i >> 1) + el;
+                const int k = k0 + 16 * kb + 4 * t + 2 * (i >> 1) + el;
                 const int n = n0 + 16 * w + g + 8 * (i & 1);
                 const int val = bf16_bits_to_int(el ? (r[i] >> 16) : (r[i] & 0xFFFFu));
                 if (n < N) q[(size_t)k * N + n] = (uint8_t)val;

@@ -95,7 +95,7 @@ def read_blob(blob, bits, K, N, group_size=128):
         words = np.ascontiguousarray(tiles[:, :, :wbytes]).view(np.uint32).reshape(strips, ktiles, 8, 32, 4)
         for p in range(8):
             reg, el = p & 3, p >> 2
-            dk = 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (reg >> 1) + el
+            dk = 16 * kb + 4 * t + 2 * (reg >> 1) + el
             dn = 16 * w + g + 8 * (reg & 1)
             vals = ((words >> np.uint32(4 * p)) & np.uint32(0xF)).astype(np.int16)
             for S in range(strips):
@@ -106,7 +106,7 @@ def read_blob(blob, bits, K, N, group_size=128):
         for r in range(2):
             for b in range(4):
                 reg, el = 2 * r + (b >> 1), b & 1
-                dk = 64 * (kb >> 2) + 16 * t + 4 * (kb & 3) + 2 * (reg >> 1) + el
+                dk = 16 * kb + 4 * t + 2 * (reg >> 1) + el
                 dn = 16 * w + g + 8 * (reg & 1)
                 for S in range(strips):
                     for T in range(ktiles):
