@@ -4,21 +4,31 @@
 // contiguous payload carrying its scales and zeros, strip after strip).  That sequence is cut into
 // equal contiguous ranges, one per CTA, so every CTA streams one contiguous byte range of HBM:
 //
-//   producer warp : one thread issues a bulk (TMA) copy per tile into a deep shared-memory ring,
-//                   completion on mbarriers; bytes in flight are bounded by the ring, not by registers.
+//   producer warp : a few lanes issue, per ring stage, one bulk (TMA) copy of several consecutive tiles
+//                   and one tiled TMA load of the activations those tiles multiply (M x 128 k per tile,
+//                   128-byte swizzled); completion on mbarriers.  Bytes in flight are bounded by the
+//                   ring, not by registers, and no consumer ever waits on a global load.
 //   consumer warps: take tiles round-robin; 128-bit shared loads, codes -> exact small-integer bf16
 //                   (q - z), contraction with the activations on the warp-level tensor-core MMA
 //                   (weights = the 16x16 operand, up to 8 tokens = the 16x8 operand: the per-weight
 //                   cost does not grow with M), fp16 scale applied in fp32 once per group.
 //
+//   reducer warp  : when the consumers finish the tiles of one strip inside this CTA's range they drop
+//                   their fp32 partials into shared memory and move on; the reducer adds them up (fixed
+//                   order), rounds to bf16 and stores y, so the consumers never wait at a strip boundary.
+//
 // A range may cut a strip (64 output columns) in two.  A CTA that holds a whole strip stores y
-// directly.  Otherwise it writes its fp32 partial to the workspace and bumps the strip's counter; the
-// CTA that arrives last adds the partials in CTA order (not arrival order) and stores y, so results
-// are deterministic and no CTA ever waits for another.  This keeps the paper's rule that partial sums
-// do not travel between workers for everything but the (at most two) cut strips of a CTA.
+// directly.  Otherwise the reducer writes the fp32 partial to the workspace and bumps the strip's
+// counter; the CTA that arrives last adds the partials in CTA order (not arrival order) and stores y, so
+// results are deterministic and no CTA ever waits for another.  The head cut of a range is published as
+// soon as it is complete (early in the kernel).  For the tail cut the reducer looks ahead: if every other
+// contributor has already published, it fetches their partials while the consumers still work, and the
+// end of the kernel is just one more add.  This keeps the paper's rule that partial sums do not travel
+// between workers for everything but the (at most two) cut strips of a CTA.
 #include "async.cuh"
 #include "common.cuh"
 #include "kernels.h"
+#include "tensormap.h"
 
 namespace tf {
 
@@ -39,26 +49,25 @@ __device__ __forceinline__ int range_owner(int tile, int total, int grid) {
 
 template <int BITS, int MT>
 __global__ void __launch_bounds__(kGemvMaxThreads, 1)
-gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a,
+gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
                    __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
-                   uint8_t* __restrict__ workspace) {
+                   int nstages, int stage_bytes, uint8_t* __restrict__ workspace) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
-    constexpr int kStageBytes = gemv_stage_bytes(BITS);
-    constexpr int nstages = gemv_stages(BITS, MT);
+    constexpr int kActOffset = kGemvActOffset;            // activations sit behind the weights of a stage
     constexpr int kTok = 8 * MT;
     constexpr int kVecPerKb = BITS == 4 ? 1 : 2;
+    constexpr int kRedWarp = kTok * kTileN;               // floats one consumer warp drops per strip segment
 
-    extern __shared__ __align__(128) uint8_t smem[];
-    // layout: [full barriers | empty barriers | flags] (1 KB) | red (consumers x kTok x 64 fp32) | ring
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // layout: barriers + flags (kGemvBarrierBytes) | red [2][consumers][kTok][64] fp32 | ring (1024-aligned stages)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 2 * kGemvMaxStages * 8);
-    volatile uint32_t* last_flag = abort_flag + 1;     // [2]: one per cut strip of this CTA
-    int* contrib_off = reinterpret_cast<int*>(smem + 1024);   // [2][kGemvMaxContrib] partial-sum offsets
-    const int nconsumers = (blockDim.x >> 5) - 1;
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + (2 * kGemvMaxStages + 4) * 8);
+    const int nconsumers = (blockDim.x >> 5) - 2;
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
-    uint8_t* ring = smem + kGemvBarrierBytes + nconsumers * kTok * kTileN * 4;
+    uint8_t* ring = smem + kGemvBarrierBytes + 2 * nconsumers * kRedWarp * 4;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int grid = gridDim.x, cta = blockIdx.x;
@@ -72,10 +81,15 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N);
 
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kGemvMaxStages);
+    const uint32_t seg_full0 = smem_u32(bars + 2 * kGemvMaxStages), seg_free0 = seg_full0 + 16;
     if (threadIdx.x == 0) {
         for (int s = 0; s < nstages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, kR);       // every tile of a chunk is released by its consumer warp
+        }
+        for (int p = 0; p < 2; ++p) {
+            mbar_init(seg_full0 + 8 * p, nconsumers);   // every consumer warp has dropped its partial
+            mbar_init(seg_free0 + 8 * p, 1);            // the reducer has read them
         }
         *abort_flag = 0;
         mbar_init_fence();
@@ -84,28 +98,147 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 
     if (warp == 0) {
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
-        // lanes 0..3 each issue every fourth chunk: one bulk copy of up to kR contiguous tiles
+        // lanes 0..3 each issue every fourth chunk: one bulk copy of up to kR contiguous tiles of one strip plus
+        // one tensor copy of the activations of those k-tiles.  Chunks never straddle a strip boundary.
         if (lane < kGemvProducerLanes && header_ok) {
-            const uint8_t* src = blob + kHeaderBytes + (size_t)t0 * kTileBytes;
-            const int nchunks = (ntiles + kR - 1) / kR;
-            for (int c = lane; c < nchunks; c += kGemvProducerLanes) {
-                const int s = c % nstages, use = c / nstages;
-                if (use >= 1 && !mbar_wait(empty0 + 8 * s, (use - 1) & 1, abort_flag, 0x100 + s)) break;
-                const int tiles_here = min(kR, ntiles - c * kR);
-                const uint32_t bytes = (uint32_t)tiles_here * kTileBytes;
-                mbar_arrive_expect_tx(full0 + 8 * s, bytes);
-                bulk_copy_g2s(smem_u32(ring + (size_t)s * kStageBytes), src + (size_t)c * kR * kTileBytes, bytes,
-                              full0 + 8 * s);
+            if (lane == 0) prefetch_tensormap(&act_map);
+            const uint32_t act_bytes = (uint32_t)M * 128u * 2u * kR;
+            int i = 0, cg = 0;
+            bool ok = true;
+            while (i < ntiles && ok) {
+                const int tile0 = t0 + i;
+                const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
+                const int seg_len = min(ntiles - i, ktiles - T0);
+                const int nchunks = (seg_len + kR - 1) / kR;
+                for (int cl = 0; cl < nchunks; ++cl, ++cg) {
+                    if (cg % kGemvProducerLanes != lane) continue;
+                    const int s = cg % nstages, use = cg / nstages;
+                    if (use >= 1 && !mbar_wait(empty0 + 8 * s, (use - 1) & 1, abort_flag, 0x100 + s)) { ok = false; break; }
+                    const int tiles_here = min(kR, seg_len - cl * kR);
+                    const uint32_t wbytes = (uint32_t)tiles_here * kTileBytes;
+                    const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
+                    mbar_arrive_expect_tx(full0 + 8 * s, wbytes + act_bytes);
+                    bulk_copy_g2s(dst, blob + kHeaderBytes + (size_t)(tile0 + cl * kR) * kTileBytes, wbytes, full0 + 8 * s);
+                    tma_load_3d(dst + kActOffset, &act_map, 0, 0, 2 * (T0 + cl * kR), full0 + 8 * s);
+                }
+                i += seg_len;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- reducer: one strip segment at a time, behind the consumers ------------------------
+        // Lane l owns output elements 4(l + 32e) .. +3 of the [token][64 n] tile (e < kVec), as float4.
+        if (header_ok) {
+            constexpr int kVec = kTok * kTileN / 128;  // float4 per lane
+            float4 pre[kVec];                          // the other contributor's partial of the tail cut, fetched early
+            bool prefetched = false;
+            int sidx = 0, i = 0;
+            bool ok = true;
+            while (i < ntiles && ok) {
+                const int tile0 = t0 + i;
+                const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
+                const int seg_len = min(ntiles - i, ktiles - T0);
+                const bool whole = seg_len == ktiles;
+                const bool is_last_seg = i + seg_len == ntiles;
+                const int p = sidx & 1;
+                const int c_first = range_owner(strip * ktiles, total_tiles, grid);
+                const int ncontrib = range_owner(strip * ktiles + ktiles - 1, total_tiles, grid) - c_first + 1;
+
+                // look ahead for the tail cut: two contributors, this CTA first, the other one already published
+                if (is_last_seg && !whole && ncontrib == 2 && c_first == cta) {
+                    uint32_t seen;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counters + strip) : "memory");
+                    if (seen == 1u) {
+                        const float4* other = reinterpret_cast<const float4*>(
+                            partials + ((size_t)(cta + 1) * 2 + 0) * (kGemvMaxM * kTileN));            // its head cut
+#pragma unroll
+                        for (int e = 0; e < kVec; ++e) pre[e] = __ldcg(other + lane + 32 * e);
+                        prefetched = true;
+                    }
+                }
+
+                ok = mbar_wait(seg_full0 + 8 * p, (sidx >> 1) & 1, abort_flag, 0x400 + p);
+                if (!ok) break;
+                // sum = partial of warp 0 + warp 1 + ... (fixed order); rows of tokens >= M hold zeros
+                float4 sum[kVec];
+#pragma unroll
+                for (int e = 0; e < kVec; ++e) sum[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int w = 0; w < nconsumers; ++w) {
+                    const float4* src = reinterpret_cast<const float4*>(red + ((size_t)p * nconsumers + w) * kRedWarp) + lane;
+#pragma unroll
+                    for (int e = 0; e < kVec; ++e) {
+                        const float4 v = src[32 * e];
+                        sum[e].x += v.x; sum[e].y += v.y; sum[e].z += v.z; sum[e].w += v.w;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(seg_free0 + 8 * p);          // consumers may reuse this buffer
+
+                const bool finish_here = whole || (prefetched && is_last_seg);
+                float4 tot[kVec];
+                bool store = finish_here;
+                if (finish_here) {
+#pragma unroll
+                    for (int e = 0; e < kVec; ++e) {
+                        tot[e] = sum[e];
+                        if (!whole) {                                    // CTA order: this CTA, then the next one
+                            tot[e].x = (0.f + sum[e].x) + pre[e].x; tot[e].y = (0.f + sum[e].y) + pre[e].y;
+                            tot[e].z = (0.f + sum[e].z) + pre[e].z; tot[e].w = (0.f + sum[e].w) + pre[e].w;
+                        }
+                    }
+                } else {
+                    // publish this CTA's partial; the last contributor to arrive adds them up in CTA order
+                    const int slot = (i == 0) ? 0 : 1;
+                    float4* mine = reinterpret_cast<float4*>(partials + ((size_t)cta * 2 + slot) * (kGemvMaxM * kTileN));
+#pragma unroll
+                    for (int e = 0; e < kVec; ++e) __stcg(mine + lane + 32 * e, sum[e]);
+                    __syncwarp();
+                    uint32_t prev = 0;
+                    if (lane == 0)
+                        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(counters + strip) : "memory");
+                    prev = __shfl_sync(0xffffffffu, prev, 0);
+                    if (prev == (uint32_t)(ncontrib - 1)) {
+#pragma unroll
+                        for (int e = 0; e < kVec; ++e) tot[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int c = 0; c < ncontrib; ++c) {
+                            const int cslot = range_start(c_first + c, total_tiles, grid) >= strip * ktiles ? 0 : 1;
+                            const float4* src = reinterpret_cast<const float4*>(
+                                partials + ((size_t)(c_first + c) * 2 + cslot) * (kGemvMaxM * kTileN)) + lane;
+#pragma unroll
+                            for (int e = 0; e < kVec; ++e) {
+                                const float4 v = __ldcg(src + 32 * e);
+                                tot[e].x += v.x; tot[e].y += v.y; tot[e].z += v.z; tot[e].w += v.w;
+                            }
+                        }
+                        store = true;
+                    }
+                }
+                if (store) {
+#pragma unroll
+                    for (int e = 0; e < kVec; ++e) {
+                        const int idx = 4 * (lane + 32 * e);
+                        const int m = idx / kTileN, n = strip * kTileN + (idx % kTileN);
+                        if (m < M && n < N) {                              // N % 8 == 0: a group of 4 columns is in or out
+                            uint2 o;
+                            o.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].x)) |
+                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].y)) << 16);
+                            o.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].z)) |
+                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].w)) << 16);
+                            *reinterpret_cast<uint2*>(y + (size_t)m * N + n) = o;
+                        }
+                    }
+                    if (!whole && lane == 0) counters[strip] = 0;          // every contributor has arrived: reset
+                }
+                i += seg_len;
+                ++sidx;
             }
         }
     } else if (header_ok) {
         // ---------------- consumers ---------------------------------------------------------------------------
-        const int cw = warp - 1, ctid = threadIdx.x - 32, cthreads = nconsumers * 32;
+        const int cw = warp - 2;
         const int g = lane >> 2, t = lane & 3;
         bool aborted = false;
-        int cut0 = -1, cut1 = -1;                      // strips this CTA holds only a part of (head, tail)
 
-        int i = 0;
+        int i = 0, sidx = 0, chunk_base = 0;
         while (i < ntiles && !aborted) {
             const int tile0 = t0 + i;
             const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
@@ -122,20 +255,15 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             // first local tile index >= i handled by this warp
             int j = i + ((cw - (i % nconsumers)) + nconsumers) % nconsumers;
             for (; j < i + seg_len; j += nconsumers) {
-                const int T = T0 + (j - i);
-                // activations of this k-tile: lane (g, t) holds token g (+8), k = 16kb + 4t .. +3 per k-block
-                uint2 av[MT][8];
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const int m = g + 8 * mt;
-                    const uint2* ap = reinterpret_cast<const uint2*>(a + (size_t)(m < M ? m : 0) * K + T * kTileK + 4 * t);
-#pragma unroll
-                    for (int kb = 0; kb < 8; ++kb) av[mt][kb] = m < M ? __ldg(ap + 4 * kb) : make_uint2(0u, 0u);
-                }
-                const int chunk = j / kR;
-                const int s = chunk % nstages;
-                if (!mbar_wait(full0 + 8 * s, (chunk / nstages) & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
-                const uint8_t* tile = ring + (size_t)s * kStageBytes + (size_t)(j - chunk * kR) * kTileBytes;
+                const int lj = j - i, cl = lj / kR, slot = lj - cl * kR;
+                const int cg = chunk_base + cl;
+                const int s = cg % nstages;
+                if (!mbar_wait(full0 + 8 * s, (cg / nstages) & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
+                const uint8_t* stage = ring + (size_t)s * stage_bytes;
+                const uint8_t* tile = stage + (size_t)slot * kTileBytes;
+                // activations of this k-tile in the stage: rows of 64 k (128 B), row index = kc * M + m with
+                // kc = 2 * slot + (kb >> 2), 16-byte chunks XOR-swizzled with (row & 7)
+                const uint8_t* acts = stage + kActOffset;
 
                 const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
                 uint32_t zg[4], zg8[4];
@@ -153,11 +281,14 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 
 #pragma unroll
                 for (int kb = 0; kb < 8; ++kb) {
-                    uint32_t b0[MT], b1[MT];
+                    uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        b0[mt] = av[mt][kb].x;
-                        b1[mt] = av[mt][kb].y;
+                        const int m = g + 8 * mt;
+                        const int row = (2 * slot + (kb >> 2)) * M + m;
+                        const int c16 = ((kb & 3) * 2 + (t >> 1)) ^ (row & 7);
+                        av[mt] = m < M ? *reinterpret_cast<const uint2*>(acts + row * 128 + c16 * 16 + (t & 1) * 8)
+                                       : make_uint2(0u, 0u);
                     }
                     uint4 wv[kVecPerKb];
 #pragma unroll
@@ -179,12 +310,17 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                             w8_word_to_regs((w & 1) ? v.w : v.y, r2, r3);
                         }
 #pragma unroll
-                        for (int mt = 0; mt < MT; ++mt) mma_bf16_16816(gacc[w][mt], r0, r1, r2, r3, b0[mt], b1[mt]);
+                        for (int mt = 0; mt < MT; ++mt)
+                            mma_bf16_16816(gacc[w][mt], r0, r1, r2, r3, av[mt].x, av[mt].y);
                     }
                 }
-                // all shared-memory reads of this stage are done: hand it back to the producer
+                // all shared-memory reads of this tile are done: hand its share of the stage back to the
+                // producer (the last tile of a short chunk also returns the shares of the missing tiles)
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * s);
+                if (lane == 0) {
+                    const int tiles_here = min(kR, seg_len - cl * kR);
+                    mbar_arrive_n(empty0 + 8 * s, slot == tiles_here - 1 ? (uint32_t)(kR - tiles_here + 1) : 1u);
+                }
 
                 // the group's scales, in fp32 (Eq. 1 / Eq. 2 factored per group)
                 const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
@@ -201,9 +337,12 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     }
                 }
             }
+            if (aborted) break;
 
-            // ---- reduce the segment over the consumer warps (fixed order) -------------------------------------
-            float* mine = red + (size_t)cw * kTok * kTileN;
+            // ---- drop this warp's partial of the segment for the reducer and move on ---------------------------
+            const int p = sidx & 1;
+            if (!mbar_wait(seg_free0 + 8 * p, ((sidx >> 1) & 1) ^ 1, abort_flag, 0x300 + p)) { aborted = true; break; }
+            float* mine = red + ((size_t)p * nconsumers + cw) * kRedWarp;       // [token][n]
 #pragma unroll
             for (int w = 0; w < 4; ++w)
 #pragma unroll
@@ -214,65 +353,11 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     mine[tok * kTileN + 16 * w + g + 8] = acc[w][mt][2];
                     mine[(tok + 1) * kTileN + 16 * w + g + 8] = acc[w][mt][3];
                 }
-            consumer_bar_sync(cthreads);
-            if (*abort_flag != 0) { aborted = true; break; }
-
-            const bool whole_strip = seg_len == ktiles;
-            const int slot = (i == 0) ? 0 : 1;
-            float* my_partial = partials + ((size_t)cta * 2 + slot) * (kGemvMaxM * kTileN);
-            for (int e = ctid; e < M * kTileN; e += cthreads) {
-                float sum = red[e];
-                for (int w = 1; w < nconsumers; ++w) sum += red[(size_t)w * kTok * kTileN + e];
-                if (whole_strip) {
-                    const int m = e / kTileN, n = strip * kTileN + (e % kTileN);
-                    if (n < N) y[(size_t)m * N + n] = __float2bfloat16_rn(sum);
-                } else {
-                    __stcg(my_partial + e, sum);               // published at the end of the kernel
-                }
-            }
-            if (!whole_strip) { if (slot == 0) cut0 = strip; else cut1 = strip; }
-            consumer_bar_sync(cthreads);                        // red is reused by the next segment
+            __syncwarp();
+            if (lane == 0) mbar_arrive(seg_full0 + 8 * p);
+            chunk_base += (seg_len + kR - 1) / kR;
             i += seg_len;
-        }
-
-        // ---- publish the partial sums of the cut strips; the last CTA to arrive for a strip adds the
-        //      partials in CTA order and stores y.  One thread per cut strip counts for the whole CTA with a
-        //      release/acquire atomic (the barrier before it orders the other threads' stores ahead of it).
-        if (!aborted && (cut0 >= 0 || cut1 >= 0)) {
-            if (ctid < 2) {
-                const int strip = ctid == 0 ? cut0 : cut1;
-                uint32_t is_last = 0;
-                if (strip >= 0) {
-                    const int c_first = range_owner(strip * ktiles, total_tiles, grid);
-                    const int c_last = range_owner(strip * ktiles + ktiles - 1, total_tiles, grid);
-                    uint32_t prev;
-                    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(counters + strip) : "memory");
-                    is_last = (prev == (uint32_t)(c_last - c_first)) ? 1u : 0u;
-                }
-                last_flag[ctid] = is_last;
-            }
-            consumer_bar_sync(cthreads);
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int strip = q == 0 ? cut0 : cut1;
-                if (strip < 0 || last_flag[q] == 0) continue;
-                const int c_first = range_owner(strip * ktiles, total_tiles, grid);
-                const int ncontrib = range_owner(strip * ktiles + ktiles - 1, total_tiles, grid) - c_first + 1;
-                // contributor c's slot: 0 if its range starts inside this strip (head), else 1 (tail)
-                for (int c = ctid; c < ncontrib; c += cthreads) {
-                    const int cslot = range_start(c_first + c, total_tiles, grid) >= strip * ktiles ? 0 : 1;
-                    contrib_off[q * kGemvMaxContrib + c] = ((c_first + c) * 2 + cslot) * (kGemvMaxM * kTileN);
-                }
-                consumer_bar_sync(cthreads);
-                for (int e = ctid; e < M * kTileN; e += cthreads) {
-                    float sum = 0.f;
-#pragma unroll 4
-                    for (int c = 0; c < ncontrib; ++c) sum += __ldcg(partials + contrib_off[q * kGemvMaxContrib + c] + e);
-                    const int m = e / kTileN, n = strip * kTileN + (e % kTileN);
-                    if (n < N) y[(size_t)m * N + n] = __float2bfloat16_rn(sum);
-                }
-                if (ctid == 0) counters[strip] = 0;            // leave the workspace ready for the next call
-            }
+            ++sidx;
         }
     }
 
@@ -299,19 +384,31 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.ktiles = K / kTileK;
     p.total_tiles = p.strips * p.ktiles;
     p.grid = p.total_tiles < sm_count ? p.total_tiles : sm_count;
-    p.consumers = kGemvMaxConsumers;
+    const int mt = M <= 8 ? 1 : 2;
+    p.consumers = mt == 1 ? kGemvMaxConsumers : 8;      // the 16-token kernel trades warps for ring depth
     const int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
     if (tiles_per_cta < p.consumers) p.consumers = tiles_per_cta < 4 ? 4 : tiles_per_cta;
-    p.threads = 32 * (p.consumers + 1);
-    const int mt = M <= 8 ? 1 : 2;
-    p.stages = gemv_stages(bits, mt);
-    p.smem_bytes = kGemvBarrierBytes + kGemvMaxConsumers * 8 * mt * kTileN * 4 + p.stages * gemv_stage_bytes(bits);
+    p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
+    const int kr = gemv_chunk_tiles(bits);
+    // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
+    p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
+    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + 2 * p.consumers * 8 * mt * kTileN * 4;
+    p.stages = (kGemvSmemBudget - fixed) / p.stage_bytes;
+    if (p.stages > kGemvMaxStages) p.stages = kGemvMaxStages;
+    p.smem_bytes = fixed + p.stages * p.stage_bytes;
     return p;
 }
 
 template <int BITS, int MT>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
+    // activations [M][K] seen as {64 k, M tokens, K/64}: one box = the M x (128 k x kR) slab of a ring stage
+    CUtensorMap map;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)M, (cuuint64_t)K / 64};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)M, (cuuint32_t)(2 * gemv_chunk_tiles(BITS))};
+    cudaError_t me = encode_bf16_map(&map, a, 3, dims, strides, box);
+    if (me != cudaSuccess) return me;
     static bool configured = false;       // the attribute is per kernel; setting it twice is harmless
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -320,8 +417,8 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
         configured = true;
     }
     gemv_stream_kernel<BITS, MT><<<p.grid, p.threads, p.smem_bytes, stream>>>(
-        static_cast<const uint8_t*>(blob), static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K,
-        N, p.ktiles, p.total_tiles, static_cast<uint8_t*>(workspace));
+        map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles,
+        p.stages, p.stage_bytes, static_cast<uint8_t*>(workspace));
     return cudaGetLastError();
 }
 

@@ -7,20 +7,16 @@ namespace tf {
 
 // ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
 constexpr int kGemvMaxConsumers = 12;
-constexpr int kGemvMaxThreads = 32 * (kGemvMaxConsumers + 1);
+constexpr int kGemvMaxThreads = 32 * (kGemvMaxConsumers + 2);   // + producer warp + reducer warp
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
 constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
 constexpr int kGemvProducerLanes = 4;         // lanes of the producer warp that issue bulk copies
 constexpr int kGemvSmemBudget = 220 * 1024;
-// A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way).
+// A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way), padded to
+// kGemvActOffset, followed by the activations of the same k-tiles.
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
-__host__ __device__ constexpr int gemv_stage_bytes(int bits) {
-    return ((bits == 4 ? 4 * 4256 : 2 * 8320) + 127) / 128 * 128;
-}
-__host__ __device__ constexpr int gemv_stages(int bits, int mt) {
-    return (kGemvSmemBudget - kGemvBarrierBytes - kGemvMaxConsumers * 8 * mt * 64 * 4) / gemv_stage_bytes(bits);
-}
+constexpr int kGemvActOffset = 17408;         // 17 x 1024 >= 4 x 4256 and >= 2 x 8320
 constexpr int kGemvMaxM = 16;
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
 // Workspace layout: [0,16) status word | [256, 256+4*512) per-strip arrival counters | partial sums
@@ -33,6 +29,7 @@ struct GemvPlan {
     int threads;       // 32 * (consumers + 1)
     int consumers;     // consumer warps
     int stages;        // ring depth
+    int stage_bytes;   // bytes of one ring stage (weights + activations)
     int smem_bytes;
     int strips, ktiles, total_tiles;
 };
