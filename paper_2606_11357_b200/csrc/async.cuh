@@ -54,6 +54,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// ---- programmatic dependent launch -------------------------------------------------------------------
+// Let the next kernel of the stream start launching now; it still has to call grid_dependency_wait()
+// before it touches anything this kernel writes.
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+// Block until every kernel this one depends on has completed and its writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- CTA pairs (clusters of two) -------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;

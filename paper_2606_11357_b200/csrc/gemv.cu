@@ -51,7 +51,8 @@ template <int BITS, int MT>
 __global__ void __launch_bounds__(kGemvMaxThreads, 1)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
                    __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
-                   int nstages, int stage_bytes, uint8_t* __restrict__ workspace) {
+                   int log2_stages, int stage_bytes, uint8_t* __restrict__ workspace) {
+    const int nstages = 1 << log2_stages;
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
@@ -95,6 +96,10 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         mbar_init_fence();
     }
     __syncthreads();
+    // Programmatic dependent launch: the next kernel on the stream may start as SMs free up.  In this kernel
+    // only the packed weights (constants) are read before grid_dependency_wait(); activations, y and the
+    // workspace are touched after it.
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
@@ -103,25 +108,34 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         if (lane < kGemvProducerLanes && header_ok) {
             if (lane == 0) prefetch_tensormap(&act_map);
             const uint32_t act_bytes = (uint32_t)M * 128u * 2u * kR;
-            int i = 0, cg = 0;
             bool ok = true;
-            while (i < ntiles && ok) {
-                const int tile0 = t0 + i;
-                const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
-                const int seg_len = min(ntiles - i, ktiles - T0);
-                const int nchunks = (seg_len + kR - 1) / kR;
-                for (int cl = 0; cl < nchunks; ++cl, ++cg) {
-                    if (cg % kGemvProducerLanes != lane) continue;
-                    const int s = cg % nstages, use = cg / nstages;
-                    if (use >= 1 && !mbar_wait(empty0 + 8 * s, (use - 1) & 1, abort_flag, 0x100 + s)) { ok = false; break; }
-                    const int tiles_here = min(kR, seg_len - cl * kR);
-                    const uint32_t wbytes = (uint32_t)tiles_here * kTileBytes;
-                    const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
-                    mbar_arrive_expect_tx(full0 + 8 * s, wbytes + act_bytes);
-                    bulk_copy_g2s(dst, blob + kHeaderBytes + (size_t)(tile0 + cl * kR) * kTileBytes, wbytes, full0 + 8 * s);
-                    tma_load_3d(dst + kActOffset, &act_map, 0, 0, 2 * (T0 + cl * kR), full0 + 8 * s);
+            // pass 0: weights of the first ring fill (before the dependency wait); pass 1: their activations,
+            // then everything else in ring order
+            for (int pass = 0; pass < 2 && ok; ++pass) {
+                if (pass == 1) grid_dependency_wait();
+                int i = 0, cg = 0;
+                while (i < ntiles && ok) {
+                    const int tile0 = t0 + i;
+                    const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
+                    const int seg_len = min(ntiles - i, ktiles - T0);
+                    const int nchunks = (seg_len + kR - 1) / kR;
+                    for (int cl = 0; cl < nchunks; ++cl, ++cg) {
+                        if (pass == 0 && cg >= nstages) break;
+                        if (cg % kGemvProducerLanes != lane) continue;
+                        const int s = cg & (nstages - 1), use = cg >> log2_stages;
+                        const int tiles_here = min(kR, seg_len - cl * kR);
+                        const uint32_t wbytes = (uint32_t)tiles_here * kTileBytes;
+                        const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
+                        if (use >= 1 && !mbar_wait(empty0 + 8 * s, (use - 1) & 1, abort_flag, 0x100 + s)) { ok = false; break; }
+                        if (pass == 0 || use >= 1) {
+                            mbar_arrive_expect_tx(full0 + 8 * s, wbytes + act_bytes);
+                            bulk_copy_g2s(dst, blob + kHeaderBytes + (size_t)(tile0 + cl * kR) * kTileBytes, wbytes, full0 + 8 * s);
+                        }
+                        if (pass == 1) tma_load_3d(dst + kActOffset, &act_map, 0, 0, 2 * (T0 + cl * kR), full0 + 8 * s);
+                    }
+                    if (pass == 0 && cg >= nstages) break;
+                    i += seg_len;
                 }
-                i += seg_len;
             }
         }
     } else if (warp == 1) {
@@ -133,6 +147,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
             bool prefetched = false;
             int sidx = 0, i = 0;
             bool ok = true;
+            grid_dependency_wait();                    // y, counters and partial sums belong to earlier kernels until now
             while (i < ntiles && ok) {
                 const int tile0 = t0 + i;
                 const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
@@ -257,13 +272,23 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
             for (; j < i + seg_len; j += nconsumers) {
                 const int lj = j - i, cl = lj / kR, slot = lj - cl * kR;
                 const int cg = chunk_base + cl;
-                const int s = cg % nstages;
-                if (!mbar_wait(full0 + 8 * s, (cg / nstages) & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
+                const int s = cg & (nstages - 1);
+                if (!mbar_wait(full0 + 8 * s, (cg >> log2_stages) & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
                 const uint8_t* stage = ring + (size_t)s * stage_bytes;
                 const uint8_t* tile = stage + (size_t)slot * kTileBytes;
                 // activations of this k-tile in the stage: rows of 64 k (128 B), row index = kc * M + m with
                 // kc = 2 * slot + (kb >> 2), 16-byte chunks XOR-swizzled with (row & 7)
                 const uint8_t* acts = stage + kActOffset;
+                const uint8_t* arow[MT][2];                    // this lane's two 128-byte rows (k 0..63, 64..127) per token tile
+                int akey[MT][2];
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int row = (2 * slot + h) * M + g + 8 * mt;
+                        arow[mt][h] = acts + row * 128 + (t & 1) * 8;
+                        akey[mt][h] = (row & 7) ^ (t >> 1);
+                    }
 
                 const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
                 uint32_t zg[4], zg8[4];
@@ -284,11 +309,10 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        const int m = g + 8 * mt;
-                        const int row = (2 * slot + (kb >> 2)) * M + m;
-                        const int c16 = ((kb & 3) * 2 + (t >> 1)) ^ (row & 7);
-                        av[mt] = m < M ? *reinterpret_cast<const uint2*>(acts + row * 128 + c16 * 16 + (t & 1) * 8)
-                                       : make_uint2(0u, 0u);
+                        // 16-byte chunk ((kb & 3) * 2 + (t >> 1)) ^ (row & 7); (kb & 3) * 2 has bit 0 clear
+                        av[mt] = g + 8 * mt < M
+                                     ? *reinterpret_cast<const uint2*>(arow[mt][kb >> 2] + ((((kb & 3) * 2) ^ akey[mt][kb >> 2]) << 4))
+                                     : make_uint2(0u, 0u);
                     }
                     uint4 wv[kVecPerKb];
 #pragma unroll
@@ -363,7 +387,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
 
     // ---------------- teardown: report, and never leave with copies in flight ------------------------------
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && (!header_ok || *abort_flag != 0)) {
+        grid_dependency_wait();
         if (!header_ok) {
             if (cta == 0) { status->code = TF_ERR_BLOB; status->detail = 1; }
         } else if (*abort_flag != 0) {
@@ -393,8 +418,10 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
     p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + 2 * p.consumers * 8 * mt * kTileN * 4;
-    p.stages = (kGemvSmemBudget - fixed) / p.stage_bytes;
-    if (p.stages > kGemvMaxStages) p.stages = kGemvMaxStages;
+    int stages = (kGemvSmemBudget - fixed) / p.stage_bytes;
+    p.log2_stages = 0;
+    while ((2 << p.log2_stages) <= stages && (2 << p.log2_stages) <= kGemvMaxStages) ++p.log2_stages;   // power of two
+    p.stages = 1 << p.log2_stages;
     p.smem_bytes = fixed + p.stages * p.stage_bytes;
     return p;
 }
@@ -416,10 +443,19 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    gemv_stream_kernel<BITS, MT><<<p.grid, p.threads, p.smem_bytes, stream>>>(
-        map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles,
-        p.stages, p.stage_bytes, static_cast<uint8_t*>(workspace));
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.grid, 1, 1);
+    cfg.blockDim = dim3(p.threads, 1, 1);
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may overlap the tail of the previous kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT>, map, static_cast<const uint8_t*>(blob),
+                              static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.log2_stages, p.stage_bytes,
+                              static_cast<uint8_t*>(workspace));
 }
 
 cudaError_t launch_gemv(int bits, const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,

@@ -28,7 +28,8 @@ struct GemvPlan {
     int grid;          // persistent CTAs
     int threads;       // 32 * (consumers + 1)
     int consumers;     // consumer warps
-    int stages;        // ring depth
+    int stages;        // ring depth (a power of two)
+    int log2_stages;
     int stage_bytes;   // bytes of one ring stage (weights + activations)
     int smem_bytes;
     int strips, ktiles, total_tiles;
