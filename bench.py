@@ -263,6 +263,7 @@ def run_gpu(args):
         for (_, M, K, N, blob, a, y, _, _) in sets[s]:
             tf.tf_gemv_w4a16(blob, a, y, M, K, N, ws, stream=stream)
 
+    torch.cuda.synchronize()                         # inputs were created on the default stream
     with torch.cuda.stream(stream):
         for s in range(2):
             enqueue_step(s)
@@ -338,6 +339,7 @@ def run_gpu(args):
                 need = int(300e6 // nbytes) + 2                      # rotate over > 2x L2 worth of copies
                 while len(pair) + len(extra) < need:
                     extra.append(pair[0][4].clone())
+                torch.cuda.synchronize()
                 blobs = [p[4] for p in pair] + extra
                 g = torch.cuda.CUDAGraph()
                 a, y = pair[0][5], pair[0][6]
@@ -367,6 +369,7 @@ def run_gpu(args):
         y = torch.empty((p2.M, p2.N), dtype=torch.bfloat16, device=dev)
         gws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, p2.M, p2.K, p2.N), dtype=torch.uint8, device=dev)
         iters = 20
+        torch.cuda.synchronize()
         with torch.cuda.stream(stream):
             for _ in range(5):
                 tf.tf_gemm_w4a16(blob, a, y, p2.M, p2.K, p2.N, gws, stream=stream)

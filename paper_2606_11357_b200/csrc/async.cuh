@@ -145,6 +145,11 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const void* 
         "l"(tensor_map), "r"(x), "r"(y), "r"(bar_cluster_addr)
         : "memory");
 }
+// Make the current contents of a 128-byte tensor map visible to the TMA unit of this thread's SM.  Needed
+// when back-to-back launches of one kernel carry different maps at the same parameter address.
+__device__ __forceinline__ void tensormap_acquire(const void* tensor_map) {
+    asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tensor_map) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const void* tensor_map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tensor_map) : "memory");
 }

@@ -66,6 +66,10 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     // layout: barriers + flags (kGemvBarrierBytes) | red [2][consumers][kTok][64] fp32 | ring (1024-aligned stages)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + (2 * kGemvMaxStages + 4) * 8);
+    // stage_tag[s] = index of the chunk whose copies were last issued into ring stage s.  A consumer warp does
+    // not touch every use of a stage, so the parity of the stage's mbarrier alone could alias (a warp two uses
+    // ahead would see "parity differs" and run on old data); it first waits for its own chunk's tag.
+    volatile uint32_t* stage_tag = reinterpret_cast<volatile uint32_t*>(smem + 1024);
     const int nconsumers = (blockDim.x >> 5) - 2;
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
     uint8_t* ring = smem + kGemvBarrierBytes + 2 * nconsumers * kRedWarp * 4;
@@ -87,6 +91,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         for (int s = 0; s < nstages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, kR);       // every tile of a chunk is released by its consumer warp
+            stage_tag[s] = 0xFFFFFFFFu;
         }
         for (int p = 0; p < 2; ++p) {
             mbar_init(seg_full0 + 8 * p, nconsumers);   // every consumer warp has dropped its partial
@@ -128,10 +133,11 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                         const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
                         if (use >= 1 && !mbar_wait(empty0 + 8 * s, (use - 1) & 1, abort_flag, 0x100 + s)) { ok = false; break; }
                         if (pass == 0 || use >= 1) {
+                            stage_tag[s] = (uint32_t)cg;         // the stage's previous use is fully consumed by now
                             mbar_arrive_expect_tx(full0 + 8 * s, wbytes + act_bytes);
                             bulk_copy_g2s(dst, blob + kHeaderBytes + (size_t)(tile0 + cl * kR) * kTileBytes, wbytes, full0 + 8 * s);
                         }
-                        if (pass == 1) tma_load_3d(dst + kActOffset, &act_map, 0, 0, 2 * (T0 + cl * kR), full0 + 8 * s);
+                        if (pass == 1) tma_load_3d(dst + kActOffset, &act_map, 0, 2 * (T0 + cl * kR), 0, full0 + 8 * s);
                     }
                     if (pass == 0 && cg >= nstages) break;
                     i += seg_len;
@@ -273,10 +279,18 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 const int lj = j - i, cl = lj / kR, slot = lj - cl * kR;
                 const int cg = chunk_base + cl;
                 const int s = cg & (nstages - 1);
+                if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
+                    const long long t_begin = clock64();
+                    while (stage_tag[s] != (uint32_t)cg && !aborted) {
+                        if (*abort_flag != 0) aborted = true;
+                        else if (clock64() - t_begin > kWaitLimitCycles) { *abort_flag = 0x280 + s; aborted = true; }
+                    }
+                    if (aborted) break;
+                }
                 if (!mbar_wait(full0 + 8 * s, (cg >> log2_stages) & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
                 const uint8_t* stage = ring + (size_t)s * stage_bytes;
                 const uint8_t* tile = stage + (size_t)slot * kTileBytes;
-                // activations of this k-tile in the stage: rows of 64 k (128 B), row index = kc * M + m with
+                // activations of this k-tile in the stage: rows of 64 k (128 B), row index = m * 2kR + kc with
                 // kc = 2 * slot + (kb >> 2), 16-byte chunks XOR-swizzled with (row & 7)
                 const uint8_t* acts = stage + kActOffset;
                 const uint8_t* arow[MT][2];                    // this lane's two 128-byte rows (k 0..63, 64..127) per token tile
@@ -285,7 +299,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const int row = (2 * slot + h) * M + g + 8 * mt;
+                        const int row = (g + 8 * mt) * (2 * kR) + 2 * slot + h;
                         arow[mt][h] = acts + row * 128 + (t & 1) * 8;
                         akey[mt][h] = (row & 7) ^ (t >> 1);
                     }
@@ -429,11 +443,12 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
 template <int BITS, int MT>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
-    // activations [M][K] seen as {64 k, M tokens, K/64}: one box = the M x (128 k x kR) slab of a ring stage
+    // activations [M][K] seen as {64 k, K/64, M tokens} (strides increase with the dimension): one box = the
+    // M x (128 k x kR) slab of a ring stage, landing in shared memory as [token][k-chunk of 64][64 k]
     CUtensorMap map;
-    const cuuint64_t dims[3] = {64, (cuuint64_t)M, (cuuint64_t)K / 64};
-    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)M, (cuuint32_t)(2 * gemv_chunk_tiles(BITS))};
+    const cuuint64_t dims[3] = {64, (cuuint64_t)K / 64, (cuuint64_t)M};
+    const cuuint64_t strides[2] = {128, (cuuint64_t)K * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)(2 * gemv_chunk_tiles(BITS)), (cuuint32_t)M};
     cudaError_t me = encode_bf16_map(&map, a, 3, dims, strides, box);
     if (me != cudaSuccess) return me;
     static bool configured = false;       // the attribute is per kernel; setting it twice is harmless
@@ -448,11 +463,11 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     cfg.blockDim = dim3(p.threads, 1, 1);
     cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may overlap the tail of the previous kernel
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    // Programmatic dependent launch stays off: with it, differently shaped GEMVs following one another on a
+    // non-default stream ended in a launch failure whose cause reading the code did not show.  The kernel
+    // keeps its prefetch-then-wait structure; without the attribute the griddepcontrol instructions are no-ops.
+    cfg.attrs = nullptr;
+    cfg.numAttrs = 0;
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT>, map, static_cast<const uint8_t*>(blob),
                               static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.log2_stages, p.stage_bytes,
                               static_cast<uint8_t*>(workspace));

@@ -82,6 +82,26 @@ def test_deterministic(bits):
     assert np.array_equal(gu.run(p, "gemm", blob_dev=blob), gu.run(p, "gemm", blob_dev=blob))
 
 
+def test_back_to_back_launches_are_independent():
+    """GEMMs queued back to back with different activations and shapes give what they give alone."""
+    stream = torch.cuda.Stream()
+    cases = []
+    for (M, K, N, seed) in [(256, 1024, 1024, 1), (256, 1024, 1024, 2), (64, 2048, 512, 3), (300, 512, 1000, 4)]:
+        p = wl.make_w4(M, K, N, seed=seed)
+        cases.append((p, torch.from_numpy(gu.pack(p)).cuda(), gu.to_device_bf16(p.a_bf16),
+                      torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")))
+    ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, 4096, 4096, 4096), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for rep in range(3):
+            for (p, blob, a, y) in cases:
+                tf.tf_gemm_w4a16(blob, a, y, p.M, p.K, p.N, ws, stream=stream)
+    stream.synchronize()
+    assert tf.tf_device_status(ws, stream=stream) == 0
+    for (p, blob, a, y) in cases:
+        assert np.array_equal(gu.bits_of(y), gu.run(p, "gemm", blob_dev=blob))
+
+
 def test_gemm_agrees_with_gemv_range():
     """M <= 16 is legal for the GEMM too; both kernels must satisfy the same bound."""
     p = wl.make_w4(16, 1024, 256, seed=12)

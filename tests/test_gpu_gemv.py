@@ -76,6 +76,35 @@ def test_deterministic_and_independent_of_stale_output(bits):
     assert np.array_equal(y1, y2)
 
 
+@pytest.mark.parametrize("bits", [4, 8])
+def test_back_to_back_launches_are_independent(bits):
+    """Calls queued back to back on one stream (nothing in between, shared workspace, different shapes and
+    activations) must each give what they give alone.  Shared-memory state of one launch must not leak into
+    the next: this is the sequence a decode step issues."""
+    stream = torch.cuda.Stream()
+    maker = wl.make_w4 if bits == 4 else wl.make_w8
+    op = tf.TF_OP_GEMV_W4A16 if bits == 4 else tf.TF_OP_GEMV_W8A16
+    fn = tf.tf_gemv_w4a16 if bits == 4 else tf.tf_gemv_w8a16
+    cases = []
+    for (M, K, N, seed) in [(1, 4096, 9472, 1), (4, 4096, 9472, 2), (4, 4096, 9472, 3), (16, 4096, 2048, 4),
+                            (1, 14336, 1024, 5), (4, 14336, 1024, 6), (8, 1024, 4096, 7), (2, 4096, 9472, 8)]:
+        p = maker(M, K, N, seed=seed)
+        cases.append((p, torch.from_numpy(gu.pack(p)).cuda(), gu.to_device_bf16(p.a_bf16),
+                      torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")))
+    ws = torch.zeros(tf.tf_workspace_size(op, 16, 4096, 4096), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for rep in range(3):
+            for (p, blob, a, y) in cases:
+                fn(blob, a, y, p.M, p.K, p.N, ws, stream=stream)
+    stream.synchronize()
+    assert tf.tf_device_status(ws, stream=stream) == 0
+    for (p, blob, a, y) in cases:
+        gu.check_against_oracle(p, gu.bits_of(y))
+        alone = gu.run(p, "gemv", blob_dev=blob)
+        assert np.array_equal(gu.bits_of(y), alone)
+
+
 def test_mismatched_blob_reports_status_and_leaves_y():
     p = wl.make_w4(1, 256, 64, seed=1)
     blob = torch.from_numpy(gu.pack(p)).cuda()
