@@ -181,6 +181,27 @@ tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
                         int M, int K, int N, void* workspace, size_t workspace_bytes,
                         void* cuda_stream);
 
+/*
+ * tf_gemv_w4a16 without a caller-provided workspace and without any allocation.  (The paper has no
+ * counterpart to this call; it exists for hosts of this library that cannot give it device memory: a
+ * plug-in in a process whose memory pool another framework owns, a thread that must stay out of the
+ * allocator, code inside a stream capture.)
+ *   Scratch (arrival counters, fp32 partial sums of strips cut between two CTAs, status word) is a fixed
+ *   array of about 1.26 MB inside the library's device image: every GPU that loads the library holds it
+ *   until the process exits.  It covers every shape tf_gemv_w4a16 accepts (1 <= M <= 16, K and N up to
+ *   32768) on devices with any SM count (at most 160 persistent CTAs are used); shapes beyond those limits
+ *   are rejected with TF_ERR_SHAPE.
+ *   The call never calls cudaMalloc, cudaFree or an allocating library routine.  The first call on a device
+ *   looks up the array's device address (one-time set-up, done with that device current): make that first
+ *   call before any stream capture.  Each call first clears, on `cuda_stream`, the part of the array that
+ *   must start at zero.  All calls share the array: calls that overlap on the GPU (different streams) race
+ *   on it, so serialise them.  The device status word is not readable through this call.
+ *   Arguments, arithmetic and results are those of tf_gemv_w4a16.
+ * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_ALIGN, TF_ERR_ARCH, TF_ERR_CUDA.
+ */
+tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_bf16,
+                               int M, int K, int N, void* cuda_stream);
+
 /* Scratch bytes the given operation needs for this shape (0 if none; 0 also if the shape
  * is illegal -- the compute call then reports TF_ERR_SHAPE). */
 size_t tf_workspace_size(int op, int M, int K, int N);

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIG
 
 EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
-           "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version")
+           "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static")
 
 
 class TileFuseError(RuntimeError):
@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
         for name in ("tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16"):
             fn = getattr(L, name)
             fn.restype, fn.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, vp, c_size, vp]
+        L.tf_gemv_w4a16_static.restype = c_int
+        L.tf_gemv_w4a16_static.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_workspace_size.restype, L.tf_workspace_size.argtypes = c_size, [c_int] * 4
         L.tf_device_status.restype, L.tf_device_status.argtypes = c_int, [vp, vp]
         L.tf_status_string.restype, L.tf_status_string.argtypes = ctypes.c_char_p, [c_int]
@@ -141,6 +143,12 @@ def _linear(name, packed, a, y, M, K, N, workspace, stream):
 def tf_gemv_w4a16(packed, a, y, M, K, N, workspace, stream=None) -> None:
     """a: bfloat16 [M,K], y: bfloat16 [M,N] CUDA tensors; asynchronous on the stream."""
     _linear("tf_gemv_w4a16", packed, a, y, M, K, N, workspace, stream)
+
+
+def tf_gemv_w4a16_static(packed, a, y, M, K, N, stream=None) -> None:
+    """tf_gemv_w4a16 for callers that cannot provide a workspace: scratch is a fixed array inside the library.
+    Calls share that array, so do not let two of them overlap on the GPU."""
+    _check("tf_gemv_w4a16_static", lib().tf_gemv_w4a16_static(_dev(packed), _dev(a), _dev(y), M, K, N, _stream(stream)))
 
 
 def tf_gemv_w8a16(packed, a, y, M, K, N, workspace, stream=None) -> None:
