@@ -48,7 +48,7 @@ __device__ __forceinline__ int range_owner(int tile, int total, int grid) {
 }  // namespace
 
 template <int BITS, int MT>
-__global__ void __launch_bounds__(kGemvMaxThreads, 1)
+__global__ void __launch_bounds__(gemv_max_threads(MT), MT == 1 ? 2 : 1)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
                    __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
                    int log2_stages, int stage_bytes, uint8_t* __restrict__ workspace) {
@@ -63,7 +63,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    // layout: barriers + flags (kGemvBarrierBytes) | red [2][consumers][kTok][64] fp32 | ring (1024-aligned stages)
+    // layout: barriers + flags (kGemvBarrierBytes) | red [consumers][kTok][64] fp32 | ring (1024-aligned stages)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + (2 * kGemvMaxStages + 4) * 8);
     // stage_tag[s] = index of the chunk whose copies were last issued into ring stage s.  A consumer warp does
@@ -72,7 +72,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     volatile uint32_t* stage_tag = reinterpret_cast<volatile uint32_t*>(smem + 1024);
     const int nconsumers = (blockDim.x >> 5) - 2;
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
-    uint8_t* ring = smem + kGemvBarrierBytes + 2 * nconsumers * kRedWarp * 4;
+    uint8_t* ring = smem + kGemvBarrierBytes + nconsumers * kRedWarp * 4;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int grid = gridDim.x, cta = blockIdx.x;
@@ -93,10 +93,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
             mbar_init(empty0 + 8 * s, kR);       // every tile of a chunk is released by its consumer warp
             stage_tag[s] = 0xFFFFFFFFu;
         }
-        for (int p = 0; p < 2; ++p) {
-            mbar_init(seg_full0 + 8 * p, nconsumers);   // every consumer warp has dropped its partial
-            mbar_init(seg_free0 + 8 * p, 1);            // the reducer has read them
-        }
+        mbar_init(seg_full0, nconsumers);               // every consumer warp has dropped its partial
+        mbar_init(seg_free0, 1);                        // the reducer has read them
         *abort_flag = 0;
         mbar_init_fence();
     }
@@ -110,7 +108,10 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
         // lanes 0..3 each issue every fourth chunk: one bulk copy of up to kR contiguous tiles of one strip plus
         // one tensor copy of the activations of those k-tiles.  Chunks never straddle a strip boundary.
-        if (lane < kGemvProducerLanes && header_ok) {
+        // A lane must see every use of the stages it serves (the parity of an mbarrier tells only one phase
+        // apart), so stage s always belongs to lane s % nlanes and nlanes divides the ring depth.
+        const int nlanes = nstages < kGemvProducerLanes ? nstages : kGemvProducerLanes;
+        if (lane < nlanes && header_ok) {
             if (lane == 0) prefetch_tensormap(&act_map);
             const uint32_t act_bytes = (uint32_t)M * 128u * 2u * kR;
             bool ok = true;
@@ -126,7 +127,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     const int nchunks = (seg_len + kR - 1) / kR;
                     for (int cl = 0; cl < nchunks; ++cl, ++cg) {
                         if (pass == 0 && cg >= nstages) break;
-                        if (cg % kGemvProducerLanes != lane) continue;
+                        if ((cg & (nlanes - 1)) != lane) continue;
                         const int s = cg & (nstages - 1), use = cg >> log2_stages;
                         const int tiles_here = min(kR, seg_len - cl * kR);
                         const uint32_t wbytes = (uint32_t)tiles_here * kTileBytes;
@@ -160,7 +161,6 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 const int seg_len = min(ntiles - i, ktiles - T0);
                 const bool whole = seg_len == ktiles;
                 const bool is_last_seg = i + seg_len == ntiles;
-                const int p = sidx & 1;
                 const int c_first = range_owner(strip * ktiles, total_tiles, grid);
                 const int ncontrib = range_owner(strip * ktiles + ktiles - 1, total_tiles, grid) - c_first + 1;
 
@@ -177,14 +177,14 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     }
                 }
 
-                ok = mbar_wait(seg_full0 + 8 * p, (sidx >> 1) & 1, abort_flag, 0x400 + p);
+                ok = mbar_wait(seg_full0, sidx & 1, abort_flag, 0x400);
                 if (!ok) break;
                 // sum = partial of warp 0 + warp 1 + ... (fixed order); rows of tokens >= M hold zeros
                 float4 sum[kVec];
 #pragma unroll
                 for (int e = 0; e < kVec; ++e) sum[e] = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int w = 0; w < nconsumers; ++w) {
-                    const float4* src = reinterpret_cast<const float4*>(red + ((size_t)p * nconsumers + w) * kRedWarp) + lane;
+                    const float4* src = reinterpret_cast<const float4*>(red + (size_t)w * kRedWarp) + lane;
 #pragma unroll
                     for (int e = 0; e < kVec; ++e) {
                         const float4 v = src[32 * e];
@@ -192,7 +192,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(seg_free0 + 8 * p);          // consumers may reuse this buffer
+                if (lane == 0) mbar_arrive(seg_free0);                  // consumers may reuse the buffer
 
                 const bool finish_here = whole || (prefetched && is_last_seg);
                 float4 tot[kVec];
@@ -378,9 +378,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
             if (aborted) break;
 
             // ---- drop this warp's partial of the segment for the reducer and move on ---------------------------
-            const int p = sidx & 1;
-            if (!mbar_wait(seg_free0 + 8 * p, ((sidx >> 1) & 1) ^ 1, abort_flag, 0x300 + p)) { aborted = true; break; }
-            float* mine = red + ((size_t)p * nconsumers + cw) * kRedWarp;       // [token][n]
+            if (!mbar_wait(seg_free0, (sidx & 1) ^ 1, abort_flag, 0x300)) { aborted = true; break; }   // previous segment read
+            float* mine = red + (size_t)cw * kRedWarp;                          // [token][n]
 #pragma unroll
             for (int w = 0; w < 4; ++w)
 #pragma unroll
@@ -392,7 +391,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     mine[(tok + 1) * kTileN + 16 * w + g + 8] = acc[w][mt][3];
                 }
             __syncwarp();
-            if (lane == 0) mbar_arrive(seg_full0 + 8 * p);
+            if (lane == 0) mbar_arrive(seg_full0);
             chunk_base += (seg_len + kR - 1) / kR;
             i += seg_len;
             ++sidx;
@@ -424,15 +423,15 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.total_tiles = p.strips * p.ktiles;
     p.grid = p.total_tiles < sm_count ? p.total_tiles : sm_count;
     const int mt = M <= 8 ? 1 : 2;
-    p.consumers = mt == 1 ? kGemvMaxConsumers : 8;      // the 16-token kernel trades warps for ring depth
+    p.consumers = gemv_max_consumers(mt);
     const int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
     if (tiles_per_cta < p.consumers) p.consumers = tiles_per_cta < 4 ? 4 : tiles_per_cta;
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
     const int kr = gemv_chunk_tiles(bits);
     // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
     p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
-    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + 2 * p.consumers * 8 * mt * kTileN * 4;
-    int stages = (kGemvSmemBudget - fixed) / p.stage_bytes;
+    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4;
+    int stages = (gemv_smem_budget(mt) - fixed) / p.stage_bytes;
     p.log2_stages = 0;
     while ((2 << p.log2_stages) <= stages && (2 << p.log2_stages) <= kGemvMaxStages) ++p.log2_stages;   // power of two
     p.stages = 1 << p.log2_stages;
@@ -454,7 +453,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     static bool configured = false;       // the attribute is per kernel; setting it twice is harmless
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kGemvSmemBudget);
+                                             gemv_smem_budget(MT));
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -463,11 +462,14 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     cfg.blockDim = dim3(p.threads, 1, 1);
     cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = stream;
-    // Programmatic dependent launch stays off: with it, differently shaped GEMVs following one another on a
-    // non-default stream ended in a launch failure whose cause reading the code did not show.  The kernel
-    // keeps its prefetch-then-wait structure; without the attribute the griddepcontrol instructions are no-ops.
-    cfg.attrs = nullptr;
-    cfg.numAttrs = 0;
+    // Programmatic dependent launch: a CTA uses less than half of an SM (shared memory, registers), so the
+    // CTAs of the next GEMV on the stream become resident while this one still runs, fill their rings with
+    // weights and then wait for this kernel to finish before they touch activations, y or the workspace.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT>, map, static_cast<const uint8_t*>(blob),
                               static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.log2_stages, p.stage_bytes,
                               static_cast<uint8_t*>(workspace));

@@ -6,13 +6,15 @@
 namespace tf {
 
 // ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
-constexpr int kGemvMaxConsumers = 12;
-constexpr int kGemvMaxThreads = 32 * (kGemvMaxConsumers + 2);   // + producer warp + reducer warp
+// Up to 8 tokens: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside this one's.
+// 9..16 tokens: twice the MMA and activation work per tile, 12 consumer warps and the whole SM.
+__host__ __device__ constexpr int gemv_max_consumers(int mt) { return mt == 1 ? 8 : 12; }
+__host__ __device__ constexpr int gemv_max_threads(int mt) { return 32 * (gemv_max_consumers(mt) + 2); }   // + producer + reducer
+__host__ __device__ constexpr int gemv_smem_budget(int mt) { return (mt == 1 ? 110 : 220) * 1024; }
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
 constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
 constexpr int kGemvProducerLanes = 4;         // lanes of the producer warp that issue bulk copies
-constexpr int kGemvSmemBudget = 220 * 1024;
 // A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way), padded to
 // kGemvActOffset, followed by the activations of the same k-tiles.
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
