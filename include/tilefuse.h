@@ -167,12 +167,17 @@ tf_status tf_gemv_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
 /*
  * Prefill-phase fused GEMM (Section 4.3 "GEMM microkernel"): 1 <= M <= 4096 tokens,
  * K, N <= 32768.  Same arguments as the GEMV.  Each packed weight tile is dequantized once
- * into shared memory as bf16 and reused by every token row of the CTA tile (the
- * dequantize-once rule of Section 4.1), then multiplied on the tcgen05 tensor cores with
- * fp32 accumulation in tensor memory.  Weights are rounded to bf16 once: w = bf16((q-z)*s).
- * Split-K partial sums (large K, few tiles) go through the workspace.
- * Errors as for the GEMV; M range 1..4096; a workspace of tf_workspace_size() bytes is
- * always required (it holds at least the status word).
+ * per CTA tile into the tensor-memory operand of the tcgen05 tensor cores as bf16 and reused by
+ * every token row of the tile (the dequantize-once rule of Section 4.1); accumulation is fp32 in
+ * tensor memory.  Weights are rounded to bf16 once: w = bf16((q-z)*s).
+ * Work is split evenly over the persistent CTAs in units of (output tile, 128-deep k-tile): an
+ * output tile whose K range is cut between CTAs is summed in fp32 through the workspace, in CTA
+ * order, by the last CTA to finish its part, so results do not depend on timing.
+ * Workspace: tf_workspace_size() bytes (tens of MB: two fp32 tile slots per CTA).  Its first
+ * 20480 bytes (status word and arrival counters) must be zero before the first call that uses
+ * it; every call leaves them zero again unless it reports an error there.  One workspace per
+ * stream: calls that run concurrently must not share one.
+ * Errors as for the GEMV; M range 1..4096.
  */
 tf_status tf_gemm_w4a16(const void* packed, const void* a_bf16, void* y_bf16,
                         int M, int K, int N, void* workspace, size_t workspace_bytes,

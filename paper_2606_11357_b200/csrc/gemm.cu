@@ -22,6 +22,10 @@
 //               packed words are stored in the register order of the 16x256b store, so a word goes from
 //               shared memory to the tensor-memory operand without any shuffle.
 //   warps 12-15 epilogue: tcgen05.ld accumulator -> bf16 -> y.
+// Work split (stream-K): the sequence of (output tile, k-tile) units is cut into equal contiguous ranges, one
+// per CTA, so all SMs finish together whatever the tile count.  A CTA that computes only part of a tile's K
+// range writes its fp32 partial accumulator to the workspace and bumps the tile's counter; the CTA that arrives
+// last adds the partials in CTA order (deterministic, nobody waits) and stores y.
 // Every mbarrier wait is bounded; on a timeout all roles leave, TMEM is freed, the status word is set.
 #include <cuda.h>
 
@@ -57,6 +61,46 @@ __host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
            kWpStages * 2 * wp_strip_bytes(bits) + 4 * kEpiWarpBytes + 512;
 }
 
+// workspace: [0,16) status | [kGemmCounterOffset, +4 * tiles) arrival counters | partial accumulators, two
+// slots of 128 x BT fp32 per CTA (head and tail of its range)
+constexpr int kGemmCounterOffset = 4096;
+constexpr int kGemmMaxTiles = 4096;            // (32768 / 128) n-tiles x (4096 / 256) token tiles
+constexpr int kGemmPartialOffset = kGemmCounterOffset + 4 * kGemmMaxTiles;
+constexpr int kGemmMaxGrid = 160;
+
+__device__ __forceinline__ int unit_start(int cta, int total, int grid) {
+    return static_cast<int>((static_cast<long long>(cta) * total) / grid);
+}
+__device__ __forceinline__ int unit_owner(int unit, int total, int grid) {
+    return static_cast<int>(((static_cast<long long>(unit) + 1) * grid - 1) / total);
+}
+
+// The CTA's unit range [u_begin, u_end) as segments of one output tile each, in processing order: the cut tile at
+// the head of the range, the cut tile at its tail, then the whole tiles.  Cut tiles go first so that the fix-up of
+// a tile shared with a neighbour runs under the main loop of a whole tile instead of at the end of the kernel.
+struct Segments {
+    int ktiles, head_tile, head_kt0, head_len, tail_tile, tail_len, first_whole, count, ncut;
+    __device__ Segments(int u_begin, int u_end, int ktiles_) : ktiles(ktiles_) {
+        head_tile = u_begin / ktiles;
+        head_kt0 = u_begin - head_tile * ktiles;
+        head_len = min(u_end - u_begin, ktiles - head_kt0);
+        if (head_len == ktiles) head_len = 0;                    // the range starts with a whole tile
+        const int u1 = u_begin + head_len;
+        const int nwhole = (u_end - u1) / ktiles;
+        first_whole = u1 / ktiles;                                // u1 is a tile boundary whenever anything follows
+        tail_tile = first_whole + nwhole;
+        tail_len = (u_end - u1) - nwhole * ktiles;
+        ncut = (head_len > 0) + (tail_len > 0);
+        count = ncut + nwhole;
+    }
+    // slot: 0 head, 1 tail, -1 whole
+    __device__ void get(int i, int& tile, int& kt0, int& len, int& slot) const {
+        if (i == 0 && head_len > 0) { tile = head_tile; kt0 = head_kt0; len = head_len; slot = 0; }
+        else if (i < ncut) { tile = tail_tile; kt0 = 0; len = tail_len; slot = 1; }
+        else { tile = first_whole + (i - ncut); kt0 = 0; len = ktiles; slot = -1; }
+    }
+};
+
 struct GemmBarriers {
     uint64_t act_full[kMaxActStages];
     uint64_t act_empty[kMaxActStages];
@@ -68,6 +112,7 @@ struct GemmBarriers {
     uint64_t acc_empty;
     uint32_t tmem_base;
     uint32_t abort_flag;
+    uint32_t last_flag;
 };
 
 __device__ __forceinline__ uint32_t bf16_dup(float v) {
@@ -99,7 +144,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = n_tiles * m_tiles;
+    const int total_units = n_tiles * m_tiles * ktiles;   // unit = (output tile, k-tile of 128)
+    const int u_begin = unit_start(blockIdx.x, total_units, gridDim.x);
+    const int u_end = unit_start(blockIdx.x + 1, total_units, gridDim.x);
+    const Segments segs(u_begin, u_end, ktiles);
     const int strips = (N + kTileN - 1) / kTileN;
     const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N);
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
@@ -138,9 +186,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             prefetch_tensormap(&act_map);
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int i = 0; i < segs.count && ok; ++i) {
+                int tile, kt0, len, slot;
+                segs.get(i, tile, kt0, len, slot);
                 const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
-                for (int ks = 0; ks < 2 * ktiles; ++ks, ++it) {
+                for (int ks = 2 * kt0; ks < 2 * (kt0 + len); ++ks, ++it) {
                     const int s = it % kStages;
                     ok = mbar_wait(smem_u32(&bars->act_empty[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x310 + s);
                     if (!ok) break;
@@ -153,11 +203,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             // ================= producer W: packed weight tiles (weights + scales + zeros in one payload) =====
             uint32_t wit = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int i = 0; i < segs.count && ok; ++i) {
+                int tile, kt0, len, slot;
+                segs.get(i, tile, kt0, len, slot);
                 const int n_tile = tile / m_tiles;
                 const int strip0 = 2 * n_tile;
                 const int nstrips = (strip0 + 1 < strips) ? 2 : 1;
-                for (int T = 0; T < ktiles; ++T, ++wit) {
+                for (int T = kt0; T < kt0 + len; ++T, ++wit) {
                     const int ws = wit % kWpStages;
                     ok = mbar_wait(smem_u32(&bars->wp_empty[ws]), ((wit / kWpStages) & 1) ^ 1, abort_flag, 0x300 + ws);
                     if (!ok) break;
@@ -172,11 +224,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             // ================= MMA issuer ==================================================================
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+            for (; tile_it < (uint32_t)segs.count && ok; ++tile_it) {
+                int tile, kt0, len, slot;
+                segs.get((int)tile_it, tile, kt0, len, slot);
                 ok = mbar_wait(smem_u32(&bars->acc_empty), (tile_it & 1) ^ 1, abort_flag, 0x400);
                 if (!ok) break;
                 tc_fence_after();
-                for (int ks = 0; ks < 2 * ktiles; ++ks, ++it) {
+                for (int ks = 0; ks < 2 * len; ++ks, ++it) {
                     const int s = it % kStages, sa = it % kAStages;
                     ok = mbar_wait(smem_u32(&bars->a_full[sa]), (it / kAStages) & 1, abort_flag, 0x410 + sa) &&
                          mbar_wait(smem_u32(&bars->act_full[s]), (it / kStages) & 1, abort_flag, 0x420 + s);
@@ -202,10 +256,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             const int g = lane >> 2;
             uint32_t wit = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int i = 0; i < segs.count && ok; ++i) {
+                int tile, kt0, len, slot;
+                segs.get(i, tile, kt0, len, slot);
                 const int n_tile = tile / m_tiles;
                 const bool strip_exists = 2 * n_tile + strip_sel < strips;
-                for (int T = 0; T < ktiles; ++T, ++wit) {
+                for (int T = kt0; T < kt0 + len; ++T, ++wit) {
                     const int ws = wit % kWpStages;
                     ok = mbar_wait(smem_u32(&bars->wp_full[ws]), (wit / kWpStages) & 1, abort_flag, 0x500 + ws);
                     if (!ok) break;
@@ -280,38 +336,109 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 }
             }
         } else if (warp >= 12) {
-            // ================= epilogue: TMEM -> bf16 -> y ===================================================
+            // ================= epilogue: TMEM -> bf16 -> y, or -> fp32 partial for a tile cut between CTAs ==========
             const int quarter = warp & 3;                     // this warp may touch TMEM lanes 32*quarter .. +31
-            uint32_t tile_it = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
-                const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
-                if (!mbar_wait(smem_u32(&bars->acc_full), tile_it & 1, abort_flag, 0x600)) break;
-                tc_fence_after();
-                // A thread reads 16 tokens of its own column n from TMEM; the warp transposes them through a
-                // private 1 KB buffer so that each thread then stores 8 consecutive columns (16 bytes) of one token.
-                const uint32_t taddr = tmem_base + (uint32_t(32 * quarter) << 16);
-                __nv_bfloat16* tbuf = reinterpret_cast<__nv_bfloat16*>(epi_buf + quarter * kEpiWarpBytes);   // [16][32]
-                const int n8 = n_tile * kBN + 32 * quarter + 8 * (lane & 3);     // first of this thread's 8 columns
-#pragma unroll 1
-                for (int c = 0; c < BT / 16; ++c) {
-                    uint32_t v[16];
-                    tmem_ld_32x32b_x16(taddr + 16 * c, v);
-                    tmem_ld_wait();
+            const int row = 32 * quarter + lane;              // this thread's weight column inside the tile
+            const uint32_t taddr = tmem_base + (uint32_t(32 * quarter) << 16);
+            __nv_bfloat16* tbuf = reinterpret_cast<__nv_bfloat16*>(epi_buf + quarter * kEpiWarpBytes);   // [16][32]
+            uint32_t* counters = reinterpret_cast<uint32_t*>(workspace + kGemmCounterOffset);
+            float* partials = reinterpret_cast<float*>(workspace + kGemmPartialOffset);
+            // 16 tokens of this thread's column -> the warp transposes them through its 1 KB buffer so that each
+            // thread stores 8 consecutive columns (16 bytes) of one token
+            auto store_chunk = [&](const float (&v)[16], int n_tile, int m_tile, int c) {
+                const int n8 = n_tile * kBN + 32 * quarter + 8 * (lane & 3);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) tbuf[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
-                    __syncwarp();
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const int tl = 8 * i + (lane >> 2);
-                        const int tok = m_tile * BT + 16 * c + tl;
-                        const uint4 d = *reinterpret_cast<const uint4*>(tbuf + tl * 32 + 8 * (lane & 3));
-                        if (tok < M && n8 < N) *reinterpret_cast<uint4*>(y + (size_t)tok * N + n8) = d;
-                    }
-                    __syncwarp();
-                }
-                tc_fence_before();
+                for (int j = 0; j < 16; ++j) tbuf[j * 32 + lane] = __float2bfloat16_rn(v[j]);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty));
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int tl = 8 * i + (lane >> 2);
+                    const int tok = m_tile * BT + 16 * c + tl;
+                    const uint4 d = *reinterpret_cast<const uint4*>(tbuf + tl * 32 + 8 * (lane & 3));
+                    if (tok < M && n8 < N) *reinterpret_cast<uint4*>(y + (size_t)tok * N + n8) = d;
+                }
+                __syncwarp();
+            };
+            uint32_t seg_it = 0;
+            for (; seg_it < (uint32_t)segs.count; ++seg_it) {
+                int tile, kt0, len, slot;
+                segs.get((int)seg_it, tile, kt0, len, slot);
+                const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
+                if (!mbar_wait(smem_u32(&bars->acc_full), seg_it & 1, abort_flag, 0x600)) break;
+                tc_fence_after();
+                if (slot < 0) {
+                    // ---- the whole K range of the tile was computed here: round and store ----------------------
+#pragma unroll 1
+                    for (int c = 0; c < BT / 16; ++c) {
+                        uint32_t r[16];
+                        float v[16];
+                        tmem_ld_32x32b_x16(taddr + 16 * c, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                        store_chunk(v, n_tile, m_tile, c);
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty));
+                } else {
+                    // ---- part of the K range: publish the fp32 partial, last arriver finishes the tile ----------
+                    // slot layout: float4 index (4 c + j) * 128 + row, so that a warp's accesses are contiguous
+                    constexpr size_t kSlotVec = (size_t)kBN * BT / 4;
+                    uint4* mine = reinterpret_cast<uint4*>(partials) + (size_t)(blockIdx.x * 2 + slot) * kSlotVec + row;
+#pragma unroll 1
+                    for (int c = 0; c < BT / 16; ++c) {
+                        uint32_t r[16];
+                        tmem_ld_32x32b_x16(taddr + 16 * c, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            __stcg(mine + (4 * c + j) * kBN, make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]));
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty));      // the accumulator is free again
+                    const int c_first = unit_owner(tile * ktiles, total_units, gridDim.x);
+                    const int ncontrib = unit_owner(tile * ktiles + ktiles - 1, total_units, gridDim.x) - c_first + 1;
+                    asm volatile("bar.sync 2, 128;" ::: "memory");               // all four epilogue warps have stored
+                    if (warp == 12 && lane == 0) {
+                        uint32_t prev;
+                        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(counters + tile) : "memory");
+                        bars->last_flag = (prev == (uint32_t)(ncontrib - 1)) ? 1u : 0u;
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                    if (*reinterpret_cast<volatile uint32_t*>(&bars->last_flag) != 0) {
+                        // sum in CTA order whoever arrived last; only the first contributor can hold a tail slot
+                        const float4* first = reinterpret_cast<const float4*>(partials) +
+                            (size_t)(c_first * 2 + (unit_start(c_first, total_units, gridDim.x) >= tile * ktiles ? 0 : 1)) * kSlotVec + row;
+                        const float4* rest = reinterpret_cast<const float4*>(partials) + (size_t)((c_first + 1) * 2) * kSlotVec + row;
+#pragma unroll 1
+                        for (int c = 0; c < BT / 16; ++c) {
+                            float4 p[4], q4[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) p[j] = __ldcg(first + (4 * c + j) * kBN);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) q4[j] = __ldcg(rest + (4 * c + j) * kBN);
+                            float v[16];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                v[4 * j] = p[j].x + q4[j].x; v[4 * j + 1] = p[j].y + q4[j].y;
+                                v[4 * j + 2] = p[j].z + q4[j].z; v[4 * j + 3] = p[j].w + q4[j].w;
+                            }
+                            for (int cc = 2; cc < ncontrib; ++cc) {
+                                const float4* src = rest + (size_t)(cc - 1) * 2 * kSlotVec;
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const float4 t4 = __ldcg(src + (4 * c + j) * kBN);
+                                    v[4 * j] += t4.x; v[4 * j + 1] += t4.y; v[4 * j + 2] += t4.z; v[4 * j + 3] += t4.w;
+                                }
+                            }
+                            store_chunk(v, n_tile, m_tile, c);
+                        }
+                        if (warp == 12 && lane == 0) counters[tile] = 0;         // leave the workspace ready for the next call
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");               // last_flag is reused by the next cut tile
+                }
             }
         }
     }
@@ -339,9 +466,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
 // ------------------------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------------------------
+static int gemm_token_tile(int M) { return M > 128 ? 256 : M > 64 ? 128 : M > 32 ? 64 : 32; }
+
 size_t gemm_workspace_bytes(int M, int K, int N) {
-    (void)M; (void)K; (void)N;
-    return 4096;                                              // status word (+ room for split-K bookkeeping)
+    (void)K; (void)N;
+    return (size_t)kGemmPartialOffset + (size_t)kGemmMaxGrid * 2 * kBN * gemm_token_tile(M) * 4;
 }
 
 namespace {
@@ -364,8 +493,9 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
         configured = true;
     }
     const int n_tiles = (N + kBN - 1) / kBN, m_tiles = (M + BT - 1) / BT;
-    const int total = n_tiles * m_tiles;
-    const int grid = total < sm_count ? total : sm_count;
+    const long long units = (long long)n_tiles * m_tiles * (K / kTileK);
+    if (sm_count > kGemmMaxGrid) sm_count = kGemmMaxGrid;
+    const int grid = units < sm_count ? (int)units : sm_count;
     gemm_kernel<BITS, BT><<<grid, kGemmThreads, gemm_smem_bytes(BITS, BT), stream>>>(
         map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K, N, K / kTileK, n_tiles, m_tiles,
         static_cast<uint8_t*>(workspace));
