@@ -4,10 +4,13 @@
 // contiguous payload carrying its scales and zeros, strip after strip).  That sequence is cut into
 // equal contiguous ranges, one per CTA, so every CTA streams one contiguous byte range of HBM:
 //
-//   producer warp : a few lanes issue, per ring stage, one bulk (TMA) copy of several consecutive tiles
+//   producer warp : one lane issues, per ring stage, one bulk (TMA) copy of several consecutive tiles
 //                   and one tiled TMA load of the activations those tiles multiply (M x 128 k per tile,
 //                   128-byte swizzled); completion on mbarriers.  Bytes in flight are bounded by the
-//                   ring, not by registers, and no consumer ever waits on a global load.
+//                   ring, not by registers, and no consumer ever waits on a global load.  One lane with
+//                   a short loop is enough: a lone lane streams 16 KB copies at the full HBM rate, while
+//                   several lanes of one warp only take turns, and every instruction of this warp
+//                   competes for issue slots with consumer warps that never idle.
 //   consumer warps: take tiles round-robin; 128-bit shared loads, codes -> exact small-integer bf16
 //                   (q - z), contraction with the activations on the warp-level tensor-core MMA
 //                   (weights = the 16x16 operand, up to 8 tokens = the 16x8 operand: the per-weight
@@ -38,6 +41,12 @@ __device__ __forceinline__ void consumer_bar_sync(int nthreads) {
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
+__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+
 __device__ __forceinline__ int range_start(int cta, int total, int grid) {
     return static_cast<int>((static_cast<long long>(cta) * total) / grid);
 }
@@ -45,14 +54,38 @@ __device__ __forceinline__ int range_owner(int tile, int total, int grid) {
     return static_cast<int>(((static_cast<long long>(tile) + 1) * grid - 1) / total);
 }
 
+// The chunks of a tile range [t0, t0 + ntiles): up to kR consecutive tiles of one strip each.  Tiles are stored
+// strip after strip, so the source pointer only ever advances.
+struct ChunkWalk {
+    int left, seg_left, T, ktiles, tile_bytes;
+    const uint8_t* src;
+    __device__ ChunkWalk(int t0, int ntiles, int ktiles_, const uint8_t* tiles, int tile_bytes_)
+        : left(ntiles), ktiles(ktiles_), tile_bytes(tile_bytes_) {
+        const int strip = t0 / ktiles;
+        T = t0 - strip * ktiles;
+        seg_left = min(ntiles, ktiles - T);
+        src = tiles + (size_t)t0 * tile_bytes;
+    }
+    __device__ bool done() const { return left == 0; }
+    __device__ void next(int kR, int& tiles_here, int& T_first, const uint8_t*& src_first) {
+        tiles_here = min(kR, seg_left);
+        T_first = T;
+        src_first = src;
+        src += (size_t)tiles_here * tile_bytes;
+        T += tiles_here;
+        seg_left -= tiles_here;
+        left -= tiles_here;
+        if (seg_left == 0) { T = 0; seg_left = min(left, ktiles); }
+    }
+};
+
 }  // namespace
 
-template <int BITS, int MT>
-__global__ void __launch_bounds__(gemv_max_threads(MT), MT == 1 ? 2 : 1)
+template <int BITS, int MT, bool FULL>
+__global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
                    __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
-                   int log2_stages, int stage_bytes, uint8_t* __restrict__ workspace) {
-    const int nstages = 1 << log2_stages;
+                   int nstages, int stage_bytes, uint8_t* __restrict__ workspace) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
@@ -106,43 +139,48 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
 
     if (warp == 0) {
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
-        // lanes 0..3 each issue every fourth chunk: one bulk copy of up to kR contiguous tiles of one strip plus
-        // one tensor copy of the activations of those k-tiles.  Chunks never straddle a strip boundary.
-        // A lane must see every use of the stages it serves (the parity of an mbarrier tells only one phase
-        // apart), so stage s always belongs to lane s % nlanes and nlanes divides the ring depth.
-        const int nlanes = nstages < kGemvProducerLanes ? nstages : kGemvProducerLanes;
-        if (lane < nlanes && header_ok) {
-            if (lane == 0) prefetch_tensormap(&act_map);
+        // One lane issues, per chunk, one bulk copy of up to kR contiguous tiles of one strip plus one tensor copy
+        // of the activations of those k-tiles.  Chunks never straddle a strip boundary.  The loop is kept to a few
+        // dozen instructions per chunk: this warp shares its scheduler with consumer warps that never idle.
+        if (lane == 0 && header_ok) {
+            prefetch_tensormap(&act_map);
             const uint32_t act_bytes = (uint32_t)M * 128u * 2u * kR;
-            bool ok = true;
-            // pass 0: weights of the first ring fill (before the dependency wait); pass 1: their activations,
-            // then everything else in ring order
-            for (int pass = 0; pass < 2 && ok; ++pass) {
-                if (pass == 1) grid_dependency_wait();
-                int i = 0, cg = 0;
-                while (i < ntiles && ok) {
-                    const int tile0 = t0 + i;
-                    const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
-                    const int seg_len = min(ntiles - i, ktiles - T0);
-                    const int nchunks = (seg_len + kR - 1) / kR;
-                    for (int cl = 0; cl < nchunks; ++cl, ++cg) {
-                        if (pass == 0 && cg >= nstages) break;
-                        if ((cg & (nlanes - 1)) != lane) continue;
-                        const int s = cg & (nstages - 1), use = cg >> log2_stages;
-                        const int tiles_here = min(kR, seg_len - cl * kR);
-                        const uint32_t wbytes = (uint32_t)tiles_here * kTileBytes;
-                        const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
-                        if (use >= 1 && !mbar_wait(empty0 + 8 * s, (use - 1) & 1, abort_flag, 0x100 + s)) { ok = false; break; }
-                        if (pass == 0 || use >= 1) {
-                            stage_tag[s] = (uint32_t)cg;         // the stage's previous use is fully consumed by now
-                            mbar_arrive_expect_tx(full0 + 8 * s, wbytes + act_bytes);
-                            bulk_copy_g2s(dst, blob + kHeaderBytes + (size_t)(tile0 + cl * kR) * kTileBytes, wbytes, full0 + 8 * s);
-                        }
-                        if (pass == 1) tma_load_3d(dst + kActOffset, &act_map, 0, 2 * (T0 + cl * kR), 0, full0 + 8 * s);
-                    }
-                    if (pass == 0 && cg >= nstages) break;
-                    i += seg_len;
+            ChunkWalk walk(t0, ntiles, ktiles, blob + kHeaderBytes, kTileBytes);
+            // first ring fill, weights only: they are constants, so they may be fetched before the dependency wait
+            int cg = 0;
+            for (; cg < nstages && !walk.done(); ++cg) {
+                int tiles_here, T;
+                const uint8_t* src;
+                walk.next(kR, tiles_here, T, src);
+                stage_tag[cg] = (uint32_t)cg;
+                mbar_arrive_expect_tx(full0 + 8 * cg, (uint32_t)tiles_here * kTileBytes + act_bytes);
+                bulk_copy_g2s(smem_u32(ring + (size_t)cg * stage_bytes), src, (uint32_t)tiles_here * kTileBytes, full0 + 8 * cg);
+            }
+            const int nfill = cg;
+            grid_dependency_wait();
+            {   // the activations of the first fill
+                ChunkWalk again(t0, ntiles, ktiles, blob + kHeaderBytes, kTileBytes);
+                for (int c = 0; c < nfill; ++c) {
+                    int tiles_here, T;
+                    const uint8_t* src;
+                    again.next(kR, tiles_here, T, src);
+                    tma_load_3d(smem_u32(ring + (size_t)c * stage_bytes) + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * c);
                 }
+            }
+            // everything else in ring order
+            int s = 0;
+            uint32_t parity = 0;
+            for (; !walk.done(); ++cg) {
+                if (!mbar_wait(empty0 + 8 * s, parity, abort_flag, 0x100 + s)) break;
+                int tiles_here, T;
+                const uint8_t* src;
+                walk.next(kR, tiles_here, T, src);
+                const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
+                stage_tag[s] = (uint32_t)cg;                 // the stage's previous use is fully consumed by now
+                mbar_arrive_expect_tx(full0 + 8 * s, (uint32_t)tiles_here * kTileBytes + act_bytes);
+                bulk_copy_g2s(dst, src, (uint32_t)tiles_here * kTileBytes, full0 + 8 * s);
+                tma_load_3d(dst + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * s);
+                if (++s == nstages) { s = 0; parity ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -260,6 +298,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         bool aborted = false;
 
         int i = 0, sidx = 0, chunk_base = 0;
+        int cg_cur = 0, s_cur = 0, use_cur = 0;         // this warp's position in the ring (chunks only move forward)
         while (i < ntiles && !aborted) {
             const int tile0 = t0 + i;
             const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
@@ -278,7 +317,10 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
             for (; j < i + seg_len; j += nconsumers) {
                 const int lj = j - i, cl = lj / kR, slot = lj - cl * kR;
                 const int cg = chunk_base + cl;
-                const int s = cg & (nstages - 1);
+                s_cur += cg - cg_cur;
+                cg_cur = cg;
+                while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
+                const int s = s_cur;
                 if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
                     const long long t_begin = clock64();
                     while (stage_tag[s] != (uint32_t)cg && !aborted) {
@@ -287,21 +329,20 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     }
                     if (aborted) break;
                 }
-                if (!mbar_wait(full0 + 8 * s, (cg >> log2_stages) & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
+                if (!mbar_wait(full0 + 8 * s, use_cur & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
                 const uint8_t* stage = ring + (size_t)s * stage_bytes;
                 const uint8_t* tile = stage + (size_t)slot * kTileBytes;
                 // activations of this k-tile in the stage: rows of 64 k (128 B), row index = m * 2kR + kc with
                 // kc = 2 * slot + (kb >> 2), 16-byte chunks XOR-swizzled with (row & 7)
-                const uint8_t* acts = stage + kActOffset;
-                const uint8_t* arow[MT][2];                    // this lane's two 128-byte rows (k 0..63, 64..127) per token tile
-                int akey[MT][2];
+                // shared address of 16-byte chunk 0 of this lane's two rows (k 0..63, 64..127) per token tile, with the
+                // swizzle key folded in: chunk c of the row is at (address ^ (c << 5))
+                uint32_t abase[MT][2];
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const int row = (g + 8 * mt) * (2 * kR) + 2 * slot + h;
-                        arow[mt][h] = acts + row * 128 + (t & 1) * 8;
-                        akey[mt][h] = (row & 7) ^ (t >> 1);
+                        abase[mt][h] = smem_u32(stage + kActOffset) + row * 128 + ((((row & 7) ^ (t >> 1))) << 4) + (t & 1) * 8;
                     }
 
                 const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
@@ -323,10 +364,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        // 16-byte chunk ((kb & 3) * 2 + (t >> 1)) ^ (row & 7); (kb & 3) * 2 has bit 0 clear
-                        av[mt] = g + 8 * mt < M
-                                     ? *reinterpret_cast<const uint2*>(arow[mt][kb >> 2] + ((((kb & 3) * 2) ^ akey[mt][kb >> 2]) << 4))
-                                     : make_uint2(0u, 0u);
+                        av[mt] = make_uint2(0u, 0u);
+                        if (g + 8 * mt < M) av[mt] = lds_v2(abase[mt][kb >> 2] ^ ((kb & 3) << 5));
                     }
                     uint4 wv[kVecPerKb];
 #pragma unroll
@@ -423,23 +462,28 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.total_tiles = p.strips * p.ktiles;
     p.grid = p.total_tiles < sm_count ? p.total_tiles : sm_count;
     const int mt = M <= 8 ? 1 : 2;
-    p.consumers = gemv_max_consumers(mt);
     const int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
+    // Long ranges amortise the start of the kernel: take the whole SM (more consumer warps, deeper ring).  Short
+    // ones gain more from the next GEMV's CTAs sitting beside this one's with their rings already full.
+    p.full = mt == 2 || tiles_per_cta >= kGemvFullFromTiles;
+    p.consumers = gemv_max_consumers(mt, p.full);
     if (tiles_per_cta < p.consumers) p.consumers = tiles_per_cta < 4 ? 4 : tiles_per_cta;
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
     const int kr = gemv_chunk_tiles(bits);
     // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
     p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4;
-    int stages = (gemv_smem_budget(mt) - fixed) / p.stage_bytes;
-    p.log2_stages = 0;
-    while ((2 << p.log2_stages) <= stages && (2 << p.log2_stages) <= kGemvMaxStages) ++p.log2_stages;   // power of two
-    p.stages = 1 << p.log2_stages;
+    int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
+    if (stages > kGemvMaxStages) stages = kGemvMaxStages;
+    // no more stages than the range has chunks
+    const int chunks = (tiles_per_cta + kr - 1) / kr + 2;
+    if (stages > chunks) stages = chunks;
+    p.stages = stages;
     p.smem_bytes = fixed + p.stages * p.stage_bytes;
     return p;
 }
 
-template <int BITS, int MT>
+template <int BITS, int MT, bool FULL>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
     // activations [M][K] seen as {64 k, K/64, M tokens} (strides increase with the dimension): one box = the
@@ -452,8 +496,8 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     if (me != cudaSuccess) return me;
     static bool configured = false;       // the attribute is per kernel; setting it twice is harmless
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             gemv_smem_budget(MT));
+        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             gemv_smem_budget(MT, FULL));
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -470,19 +514,21 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT>, map, static_cast<const uint8_t*>(blob),
-                              static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.log2_stages, p.stage_bytes,
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL>, map, static_cast<const uint8_t*>(blob),
+                              static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
                               static_cast<uint8_t*>(workspace));
 }
 
 cudaError_t launch_gemv(int bits, const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                         int N, void* workspace, cudaStream_t stream) {
     if (bits == 4) {
-        return M <= 8 ? launch_one<4, 1>(p, blob, a, y, M, K, N, workspace, stream)
-                      : launch_one<4, 2>(p, blob, a, y, M, K, N, workspace, stream);
+        if (M > 8) return launch_one<4, 2, true>(p, blob, a, y, M, K, N, workspace, stream);
+        return p.full ? launch_one<4, 1, true>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<4, 1, false>(p, blob, a, y, M, K, N, workspace, stream);
     }
-    return M <= 8 ? launch_one<8, 1>(p, blob, a, y, M, K, N, workspace, stream)
-                  : launch_one<8, 2>(p, blob, a, y, M, K, N, workspace, stream);
+    if (M > 8) return launch_one<8, 2, true>(p, blob, a, y, M, K, N, workspace, stream);
+    return p.full ? launch_one<8, 1, true>(p, blob, a, y, M, K, N, workspace, stream)
+                  : launch_one<8, 1, false>(p, blob, a, y, M, K, N, workspace, stream);
 }
 
 }  // namespace tf

@@ -6,15 +6,17 @@
 namespace tf {
 
 // ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
-// Up to 8 tokens: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside this one's.
+// Up to 8 tokens, short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside
+// this one's and fill their rings while it finishes.  Up to 8 tokens, long ranges: the whole SM, 14 consumer
+// warps and a ring deep enough to keep HBM busy while 14 tiles are being consumed.
 // 9..16 tokens: twice the MMA and activation work per tile, 12 consumer warps and the whole SM.
-__host__ __device__ constexpr int gemv_max_consumers(int mt) { return mt == 1 ? 8 : 12; }
-__host__ __device__ constexpr int gemv_max_threads(int mt) { return 32 * (gemv_max_consumers(mt) + 2); }   // + producer + reducer
-__host__ __device__ constexpr int gemv_smem_budget(int mt) { return (mt == 1 ? 110 : 220) * 1024; }
+__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 14 : 8) : 12; }
+__host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
+__host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
+constexpr int kGemvFullFromTiles = 96;        // tiles per CTA from which up to 8 tokens use the whole-SM configuration
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
 constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
-constexpr int kGemvProducerLanes = 4;         // lanes of the producer warp that issue bulk copies
 // A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way), padded to
 // kGemvActOffset, followed by the activations of the same k-tiles.
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
@@ -30,8 +32,8 @@ struct GemvPlan {
     int grid;          // persistent CTAs
     int threads;       // 32 * (consumers + 1)
     int consumers;     // consumer warps
-    int stages;        // ring depth (a power of two)
-    int log2_stages;
+    int stages;        // ring depth
+    bool full;         // whole-SM configuration
     int stage_bytes;   // bytes of one ring stage (weights + activations)
     int smem_bytes;
     int strips, ktiles, total_tiles;
