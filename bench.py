@@ -256,7 +256,8 @@ def run_gpu(args):
                 y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
                 y_host = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
                 calls.append((s, M, K, N, blob, a, y, a_host, y_host))
-    sets = [[c for c in calls if c[0] == s] for s in range(2)]
+    # one decode step per batch size: for each M, the four layer shapes in turn (as a model runs them)
+    sets = [[c for M in GEMV_MS for c in calls if c[0] == s and c[1] == M] for s in range(2)]
     launches_per_step = len(sets[0])
 
     def enqueue_step(s):
@@ -403,7 +404,7 @@ def run_gpu(args):
         "warmup": 2 * replays_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "cfg1 decode GEMV sweep: Llama-3-8B layer shapes 4096x4096, 4096x1024, 4096x14336, "
-                               "14336x4096 at M=1,4,16 (12 tf_gemv_w4a16 calls per step)",
+                               "14336x4096 for M=1, then M=4, then M=16 (12 tf_gemv_w4a16 calls per step)",
                    "l2": "inputs larger than L2: two alternating sets of 12 weight copies, 432 MB in rotation",
                    "bytes_per_step": step_bytes, "launch": "CUDA graph replay of two steps"},
         "clocks": clocks,

@@ -258,15 +258,29 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     if (prev == (uint32_t)(ncontrib - 1)) {
 #pragma unroll
                         for (int e = 0; e < kVec; ++e) tot[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int c = 0; c < ncontrib; ++c) {
-                            const int cslot = range_start(c_first + c, total_tiles, grid) >= strip * ktiles ? 0 : 1;
-                            const float4* src = reinterpret_cast<const float4*>(
-                                partials + ((size_t)(c_first + c) * 2 + cslot) * (kGemvMaxM * kTileN)) + lane;
+                        // The sum runs in CTA order, but the loads of several contributors are issued together: one
+                        // L2 round trip per batch instead of one per contributor.  Rows of tokens >= M are never read.
+                        constexpr int kBatch = MT == 1 ? 4 : 2;
+                        for (int c0 = 0; c0 < ncontrib; c0 += kBatch) {
+                            float4 v[kBatch][kVec];
 #pragma unroll
-                            for (int e = 0; e < kVec; ++e) {
-                                const float4 v = __ldcg(src + 32 * e);
-                                tot[e].x += v.x; tot[e].y += v.y; tot[e].z += v.z; tot[e].w += v.w;
+                            for (int b = 0; b < kBatch; ++b) {
+                                const int c = c0 + b;
+                                const int cslot = range_start(c_first + c, total_tiles, grid) >= strip * ktiles ? 0 : 1;
+                                const float4* src = reinterpret_cast<const float4*>(
+                                    partials + ((size_t)(c_first + c) * 2 + cslot) * (kGemvMaxM * kTileN)) + lane;
+#pragma unroll
+                                for (int e = 0; e < kVec; ++e) {
+                                    v[b][e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    if (c < ncontrib && 2 * e < M) v[b][e] = __ldcg(src + 32 * e);
+                                }
                             }
+#pragma unroll
+                            for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+                                for (int e = 0; e < kVec; ++e) {
+                                    tot[e].x += v[b][e].x; tot[e].y += v[b][e].y; tot[e].z += v[b][e].z; tot[e].w += v[b][e].w;
+                                }
                         }
                         store = true;
                     }
@@ -498,6 +512,12 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              gemv_smem_budget(MT, FULL));
+        if (e != cudaSuccess) return e;
+        // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
+        // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
+        // consecutive GEMVs of different shapes could not share an SM.
+        e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
     }
