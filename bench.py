@@ -430,8 +430,11 @@ def run_profile_case(args):
     from paper_2606_11357_b200 import workloads as wl
     torch.cuda.set_device(0)
     kind, bits = args.profile_case.split("_")
+    big = bits.endswith("big")
     bits = int(bits[1])
-    if kind == "gemv":
+    if kind == "gemv" and big:
+        prob = wl.config4_gemv()
+    elif kind == "gemv":
         prob = (wl.config1(args.profile_m or 1, 4096, 14336) if bits == 4 else wl.config3_gemv())
     else:
         prob = (wl.config2(args.profile_m or 2048) if bits == 4 else wl.config3_gemm())
@@ -461,7 +464,7 @@ def main(argv=None):
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--skip-gemm", action="store_true", help="leave out the prefill GEMM section")
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline")
-    ap.add_argument("--profile-case", choices=["gemv_w4", "gemv_w8", "gemm_w4", "gemm_w8"], default=None,
+    ap.add_argument("--profile-case", choices=["gemv_w4", "gemv_w4big", "gemv_w8", "gemm_w4", "gemm_w8"], default=None,
                     help="run --steps launches of one kernel on one case and exit (for ncu captures)")
     ap.add_argument("--profile-m", type=int, default=0, help="token count for --profile-case")
     args = ap.parse_args(argv)

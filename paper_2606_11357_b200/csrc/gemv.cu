@@ -479,7 +479,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     const int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
     // Long ranges amortise the start of the kernel: take the whole SM (more consumer warps, deeper ring).  Short
     // ones gain more from the next GEMV's CTAs sitting beside this one's with their rings already full.
-    p.full = mt == 2 || tiles_per_cta >= kGemvFullFromTiles;
+    p.full = mt == 2 || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= kGemvFullFromBytes;
     p.consumers = gemv_max_consumers(mt, p.full);
     if (tiles_per_cta < p.consumers) p.consumers = tiles_per_cta < 4 ? 4 : tiles_per_cta;
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp

@@ -7,13 +7,13 @@ namespace tf {
 
 // ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
 // Up to 8 tokens, short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside
-// this one's and fill their rings while it finishes.  Up to 8 tokens, long ranges: the whole SM, 14 consumer
-// warps and a ring deep enough to keep HBM busy while 14 tiles are being consumed.
+// this one's and fill their rings while it finishes.  Up to 8 tokens, long ranges: the whole SM, 12 consumer
+// warps and a ring deep enough to keep HBM busy while 12 tiles are being consumed.
 // 9..16 tokens: twice the MMA and activation work per tile, 12 consumer warps and the whole SM.
-__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 14 : 8) : 12; }
+__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 12; }
 __host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
-constexpr int kGemvFullFromTiles = 96;        // tiles per CTA from which up to 8 tokens use the whole-SM configuration
+constexpr int kGemvFullFromBytes = 384 * 1024; // packed bytes per CTA from which up to 8 tokens use the whole-SM configuration
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
 constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
