@@ -393,6 +393,39 @@ def run_gpu(args):
                              "frac": tfl / peaks["bf16_tflops"], "peak_kind": f"{peak_kind} (burst, cuBLAS bf16)",
                              "traffic": traffic.get("gemm_w4_cfg2_dram_bytes_per_launch")}}
 
+    # ---- library kernels on the same sizes, as context (not part of the path, not a target) ----------------
+    ceilings = None
+    if rank == 0 and not args.skip_gemm:
+        ceilings = {}
+        with torch.cuda.stream(stream):
+            # bf16 x bf16 library GEMM on the config-2 shape (weights already full precision in HBM)
+            w_full = torch.randn((p2.K, p2.N), device=dev).to(torch.bfloat16)
+            for _ in range(3):
+                torch.matmul(a, w_full)
+            stream.synchronize()
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record(stream)
+            for _ in range(10):
+                torch.matmul(a, w_full)
+            c1.record(stream)
+            stream.synchronize()
+            ceilings["matmul_bf16_cfg2_tflops"] = round(2.0 * p2.M * p2.K * p2.N / (c0.elapsed_time(c1) * 1e3 / 10) / 1e6, 1)
+            del w_full
+            # a read-only pass (library reduction) over 512 MB: what a kernel that only reads can reach
+            src = torch.empty(128 * 1024 * 1024, dtype=torch.int32, device=dev)
+            src.zero_()
+            for _ in range(2):
+                src.sum()
+            stream.synchronize()
+            c0.record(stream)
+            for _ in range(5):
+                src.sum()
+            c1.record(stream)
+            stream.synchronize()
+            ceilings["read_only_pass_gbs"] = round(src.numel() * 4 / (c0.elapsed_time(c1) * 1e3 / 5) / 1e3, 1)
+            del src
+        ceilings["note"] = "torch library kernels, same process, context only"
+
     if rank != 0:
         return 0
     cpu_baseline = None
@@ -418,6 +451,7 @@ def run_gpu(args):
         "cpu_baseline": cpu_baseline,
         "per_shape": per_shape,
         "gemm": gemm,
+        "ceilings": ceilings,
     }
     print(json.dumps(line), flush=True)
     return 0

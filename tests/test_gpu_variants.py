@@ -1,0 +1,55 @@
+"""Variants of the setup the paper also describes (Section 2.1: per-channel W8A16 scales; group sizes above
+128; token counts between the decode and prefill ranges): same kernels, same acceptance rule."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tilefuse_oracle as orc
+from paper_2606_11357_b200 import binding as tf
+from paper_2606_11357_b200 import workloads as wl
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("kind,M", [("gemv", 1), ("gemv", 16), ("gemm", 40), ("gemm", 300)])
+def test_w8_per_channel_scales(kind, M):
+    """group_size == K: one scale per output column."""
+    K, N = 1024, 712
+    p = wl.make_w8(M, K, N, seed=500 + M, group_size=K)
+    assert p.scales_f16.shape == (1, N)
+    gu.check_against_oracle(p, gu.run(p, kind))
+
+
+@pytest.mark.parametrize("kind,M,g", [("gemv", 3, 256), ("gemv", 9, 512), ("gemm", 130, 256), ("gemm", 64, 1536)])
+def test_w4_group_sizes_above_the_tile(kind, M, g):
+    K, N = 1536, 328
+    p = wl.make_w4(M, K, N, seed=600 + M, group_size=g)
+    gu.check_against_oracle(p, gu.run(p, kind))
+
+
+def test_unpack_with_group_256_is_bit_exact():
+    K, N, g = 1024, 136, 256
+    p = wl.make_w4(1, K, N, seed=77, group_size=g)
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    q = torch.full((K, N), 0xEE, dtype=torch.uint8, device="cuda")
+    z = torch.full((K // g, N), 0xEE, dtype=torch.uint8, device="cuda")
+    s = torch.zeros((K // g, N), dtype=torch.float16, device="cuda")
+    tf.tf_unpack_w4(blob, q, z, s, K, N, g)
+    torch.cuda.synchronize()
+    assert np.array_equal(q.cpu().numpy(), orc.unpack_awq(p.qweight))
+    assert np.array_equal(z.cpu().numpy(), orc.unpack_awq(p.qzeros))
+    assert np.array_equal(s.cpu().numpy().view(np.uint16), p.scales_f16.view(np.uint16))
+
+
+@pytest.mark.parametrize("M", [17, 33, 100, 129, 255])
+def test_medium_token_counts_through_the_gemm(M):
+    """Between the decode (<= 16) and prefill ranges the GEMM entry point applies, with smaller token tiles."""
+    p = wl.make_w4(M, 2048, 1096, seed=700 + M)
+    gu.check_against_oracle(p, gu.run(p, "gemm"))
+
+
+def test_illegal_group_sizes_are_rejected():
+    assert tf.tf_packed_size(4, 1024, 64, 64) == 0          # below the tile's k-extent
+    assert tf.tf_packed_size(4, 1024, 64, 384) == 0         # does not divide K
+    assert tf.tf_packed_size(8, 1024, 64, 1024) > 0
