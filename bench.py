@@ -412,7 +412,7 @@ def run_gpu(args):
             ceilings["matmul_bf16_cfg2_tflops"] = round(2.0 * p2.M * p2.K * p2.N / (c0.elapsed_time(c1) * 1e3 / 10) / 1e6, 1)
             del w_full
             # a read-only pass (library reduction) over 512 MB: what a kernel that only reads can reach
-            src = torch.empty(128 * 1024 * 1024, dtype=torch.int32, device=dev)
+            src = torch.empty(128 * 1024 * 1024, dtype=torch.float32, device=dev)
             src.zero_()
             for _ in range(2):
                 src.sum()
