@@ -79,13 +79,33 @@ struct ChunkWalk {
     }
 };
 
+// fp32 [token][64 n] tile held as float4 per lane (element 4 (lane + 32 e)) -> bf16 -> y; rows >= M and columns >= N
+// are not written (N % 8 == 0: a group of 4 columns is in or out)
+template <int kVec>
+__device__ __forceinline__ void store_strip(__nv_bfloat16* y, const float4 (&tot)[kVec], int strip, int M, int N, int lane) {
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) {
+        const int idx = 4 * (lane + 32 * e);
+        const int m = idx / kTileN, n = strip * kTileN + (idx % kTileN);
+        if (m < M && n < N) {
+            uint2 o;
+            o.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].x)) |
+                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].y)) << 16);
+            o.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].z)) |
+                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].w)) << 16);
+            *reinterpret_cast<uint2*>(y + (size_t)m * N + n) = o;
+        }
+    }
+}
+
 }  // namespace
 
-template <int BITS, int MT, bool FULL>
+template <int BITS, int MT, bool FULL, bool CL>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
                    __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
-                   int nstages, int stage_bytes, uint8_t* __restrict__ workspace) {
+                   int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes,
+                   uint8_t* __restrict__ workspace) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
@@ -105,12 +125,24 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     volatile uint32_t* stage_tag = reinterpret_cast<volatile uint32_t*>(smem + 1024);
     const int nconsumers = (blockDim.x >> 5) - 2;
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
-    uint8_t* ring = smem + kGemvBarrierBytes + nconsumers * kRedWarp * 4;
+    // xred [csize][xslot]: in cluster mode, the partials other CTAs of the cluster send to the finisher of a strip
+    uint8_t* xred = smem + kGemvBarrierBytes + nconsumers * kRedWarp * 4;
+    uint8_t* ring = xred + ((CL && csize > 1 ? csize * xslot_bytes : 0) + 1023) / 1024 * 1024;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int grid = gridDim.x, cta = blockIdx.x;
-    const int t0 = range_start(cta, total_tiles, grid);
-    const int ntiles = range_start(cta + 1, total_tiles, grid) - t0;
+    const int cta = blockIdx.x;
+    // "Contributor space": the CTAs that split one pool of tiles evenly among themselves.  Global mode: all CTAs
+    // of the grid over all tiles.  Cluster mode: the CTAs of one cluster over the whole strips that cluster owns,
+    // so that a strip is only ever shared inside a cluster and can be summed through distributed shared memory.
+    int cn = gridDim.x, crank = cta, cbase = 0, ctiles = total_tiles;
+    if (CL && csize > 1) {
+        const int q = cta / csize, strips = total_tiles / ktiles;
+        const int s0 = (int)(((long long)q * strips) / nclusters), s1 = (int)(((long long)(q + 1) * strips) / nclusters);
+        cn = csize; crank = cta - q * csize; cbase = s0 * ktiles; ctiles = (s1 - s0) * ktiles;
+    }
+    const int t0 = cbase + range_start(crank, ctiles, cn);
+    const int ntiles = cbase + range_start(crank + 1, ctiles, cn) - t0;
+    int fin_strip = -1, fin_first = 0;          // cluster mode: the strip this CTA finishes after the cluster barrier
 
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
     uint32_t* counters = reinterpret_cast<uint32_t*>(workspace + kGemvCounterOffset);
@@ -199,11 +231,12 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 const int seg_len = min(ntiles - i, ktiles - T0);
                 const bool whole = seg_len == ktiles;
                 const bool is_last_seg = i + seg_len == ntiles;
-                const int c_first = range_owner(strip * ktiles, total_tiles, grid);
-                const int ncontrib = range_owner(strip * ktiles + ktiles - 1, total_tiles, grid) - c_first + 1;
+                const int c_first = range_owner(strip * ktiles - cbase, ctiles, cn);
+                const int c_last = range_owner(strip * ktiles + ktiles - 1 - cbase, ctiles, cn);
+                const int ncontrib = c_last - c_first + 1;
 
                 // look ahead for the tail cut: two contributors, this CTA first, the other one already published
-                if (is_last_seg && !whole && ncontrib == 2 && c_first == cta) {
+                if ((!CL || csize == 1) && is_last_seg && !whole && ncontrib == 2 && c_first == cta) {
                     uint32_t seen;
                     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counters + strip) : "memory");
                     if (seen == 1u) {
@@ -244,6 +277,16 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                             tot[e].z = (0.f + sum[e].z) + pre[e].z; tot[e].w = (0.f + sum[e].w) + pre[e].w;
                         }
                     }
+                } else if (CL && csize > 1) {
+                    // cluster mode: hand the partial to the CTA that holds the strip's last tile (maybe this one);
+                    // it adds the slots up in rank order after the cluster barrier at the end of the kernel
+                    const uint32_t remote = map_to_cta(smem_u32(xred + (size_t)crank * xslot_bytes), (uint32_t)c_last);
+#pragma unroll
+                    for (int e = 0; e < kVec; ++e)
+                        if (2 * e < M)
+                            asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote + (lane + 32 * e) * 16),
+                                         "f"(sum[e].x), "f"(sum[e].y), "f"(sum[e].z), "f"(sum[e].w) : "memory");
+                    if (c_last == crank) { fin_strip = strip; fin_first = c_first; }
                 } else {
                     // publish this CTA's partial; the last contributor to arrive adds them up in CTA order
                     const int slot = (i == 0) ? 0 : 1;
@@ -266,7 +309,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
 #pragma unroll
                             for (int b = 0; b < kBatch; ++b) {
                                 const int c = c0 + b;
-                                const int cslot = range_start(c_first + c, total_tiles, grid) >= strip * ktiles ? 0 : 1;
+                                const int cslot = range_start(c_first + c, total_tiles, cn) >= strip * ktiles ? 0 : 1;
                                 const float4* src = reinterpret_cast<const float4*>(
                                     partials + ((size_t)(c_first + c) * 2 + cslot) * (kGemvMaxM * kTileN)) + lane;
 #pragma unroll
@@ -286,20 +329,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     }
                 }
                 if (store) {
-#pragma unroll
-                    for (int e = 0; e < kVec; ++e) {
-                        const int idx = 4 * (lane + 32 * e);
-                        const int m = idx / kTileN, n = strip * kTileN + (idx % kTileN);
-                        if (m < M && n < N) {                              // N % 8 == 0: a group of 4 columns is in or out
-                            uint2 o;
-                            o.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].x)) |
-                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].y)) << 16);
-                            o.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].z)) |
-                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(tot[e].w)) << 16);
-                            *reinterpret_cast<uint2*>(y + (size_t)m * N + n) = o;
-                        }
-                    }
-                    if (!whole && lane == 0) counters[strip] = 0;          // every contributor has arrived: reset
+                    store_strip<kVec>(y, tot, strip, M, N, lane);
+                    if (!whole && (!CL || csize == 1) && lane == 0) counters[strip] = 0;          // every contributor has arrived: reset
                 }
                 i += seg_len;
                 ++sidx;
@@ -451,8 +482,32 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         }
     }
 
-    // ---------------- teardown: report, and never leave with copies in flight ------------------------------
+    // ---------------- cluster mode: finish the strip whose last tile this CTA holds -----------------------------
     __syncthreads();
+    if (CL && csize > 1) {
+        // Every CTA of the cluster gets here (all waits above are bounded).  After the barrier the partials the
+        // other CTAs stored into this CTA's slots are visible, and nobody touches another CTA's memory again.
+        cluster_sync_all();
+        if (warp == 1 && fin_strip >= 0 && header_ok && *abort_flag == 0) {
+            constexpr int kVec = kTok * kTileN / 128;
+            float4 tot[kVec];
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) tot[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c = fin_first; c <= crank; ++c) {                     // rank order, as in global mode
+                if (range_start(c + 1, ctiles, cn) == range_start(c, ctiles, cn)) continue;   // empty range: no partial
+                const float4* src = reinterpret_cast<const float4*>(xred + (size_t)c * xslot_bytes) + lane;
+#pragma unroll
+                for (int e = 0; e < kVec; ++e)
+                    if (2 * e < M) {
+                        const float4 v = src[32 * e];
+                        tot[e].x += v.x; tot[e].y += v.y; tot[e].z += v.z; tot[e].w += v.w;
+                    }
+            }
+            store_strip<kVec>(y, tot, fin_strip, M, N, lane);
+        }
+    }
+
+    // ---------------- teardown: report, and never leave with copies in flight ------------------------------
     if (threadIdx.x == 0 && (!header_ok || *abort_flag != 0)) {
         grid_dependency_wait();
         if (!header_ok) {
@@ -468,7 +523,41 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     }
 }
 
-// Launch geometry: one persistent CTA per SM (fewer when there are fewer tiles than SMs).
+// How many clusters of `csize` whole-SM CTAs the device can hold at once (asked once per device; half-SM CTAs fit
+// at least as often).  0 if the question fails: cluster mode is then not used.
+static int max_resident_clusters(int csize) {
+    static int cached[kGemvMaxDevices][4];      // [device][log2 csize], 0 = not asked yet, -1 = failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kGemvMaxDevices) return 0;
+    const int slot = csize == 2 ? 1 : csize == 4 ? 2 : 3;
+    if (cached[dev][slot] == 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(csize * 32, 1, 1);
+        cfg.blockDim = dim3(gemv_max_threads(1, true), 1, 1);
+        cfg.dynamicSmemBytes = gemv_smem_budget(1, true);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             gemv_smem_budget(1, true));
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, true, true>, &cfg);
+        if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
+        cached[dev][slot] = n > 0 ? n : -1;
+    }
+    return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
+}
+
+// Launch geometry.  Global mode: one persistent CTA per SM (fewer when there are fewer tiles than SMs), all tiles
+// cut into equal ranges; a strip cut between CTAs is summed through the workspace.  Cluster mode: clusters of 2, 4
+// or 8 CTAs, each cluster owning whole strips and cutting its tiles into equal ranges among its CTAs; a cut strip
+// is summed through distributed shared memory, which is several microseconds shorter than the workspace hand-over
+// (partial to L2, atomic, loads by the last arriver).  A kernel that contains cluster instructions starts about
+// 0.7 us later than one that does not, even when launched without clusters, and a cluster launch overlaps less
+// with its neighbours on the stream, so cluster mode has instantiations of its own and is taken only for short
+// ranges, where the hand-over dominates the call.
 GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     GemvPlan p;
     p.strips = (N + kTileN - 1) / kTileN;
@@ -476,7 +565,29 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.total_tiles = p.strips * p.ktiles;
     p.grid = p.total_tiles < sm_count ? p.total_tiles : sm_count;
     const int mt = M <= 8 ? 1 : 2;
-    const int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
+    int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
+    p.cluster = 1;
+    p.nclusters = 0;
+    int best_t = 0;
+    for (int c = 2; c <= 8; c *= 2) {
+        int maxc = max_resident_clusters(c);
+        if (maxc > sm_count / c) maxc = sm_count / c;
+        if (maxc < 1) continue;
+        const int j = (p.strips + maxc - 1) / maxc;                 // whole strips per cluster, at most
+        const int ncl = (p.strips + j - 1) / j;
+        const int t = (j * p.ktiles + c - 1) / c;                   // longest range of a CTA
+        if (p.cluster == 1 || t < best_t) { p.cluster = c; p.nclusters = ncl; best_t = t; }
+    }
+    // worth it for short ranges only (there the hand-over dominates the call), and only if the longest range stays
+    // within one round of the consumer warps or close to the evenly split one
+    const int one_round = gemv_max_consumers(mt, mt == 2);
+    if (p.cluster > 1 && tiles_per_cta <= 32 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
+        p.grid = p.nclusters * p.cluster;
+        tiles_per_cta = best_t;
+    } else {
+        p.cluster = 1;
+        p.nclusters = 0;
+    }
     // Long ranges amortise the start of the kernel: take the whole SM (more consumer warps, deeper ring).  Short
     // ones gain more from the next GEMV's CTAs sitting beside this one's with their rings already full.
     p.full = mt == 2 || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= kGemvFullFromBytes;
@@ -486,7 +597,10 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     const int kr = gemv_chunk_tiles(bits);
     // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
     p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
-    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4;
+    // cluster mode: one slot per CTA of the cluster for the rows of real tokens (two token rows = 512 bytes)
+    p.xslot_bytes = p.cluster > 1 ? ((M + 1) / 2) * 512 : 0;
+    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4 +
+                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024;
     int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
     if (stages > kGemvMaxStages) stages = kGemvMaxStages;
     // no more stages than the range has chunks
@@ -497,7 +611,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     return p;
 }
 
-template <int BITS, int MT, bool FULL>
+template <int BITS, int MT, bool FULL, bool CL>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
     // activations [M][K] seen as {64 k, K/64, M tokens} (strides increase with the dimension): one box = the
@@ -510,13 +624,13 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     if (me != cudaSuccess) return me;
     static bool configured = false;       // the attribute is per kernel; setting it twice is harmless
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              gemv_smem_budget(MT, FULL));
         if (e != cudaSuccess) return e;
         // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
         // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
         // consecutive GEMVs of different shapes could not share an SM.
-        e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -529,26 +643,39 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     // Programmatic dependent launch: a CTA uses less than half of an SM (shared memory, registers), so the
     // CTAs of the next GEMV on the stream become resident while this one still runs, fill their rings with
     // weights and then wait for this kernel to finish before they touch activations, y or the workspace.
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL>, map, static_cast<const uint8_t*>(blob),
+    if (p.cluster > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL>, map, static_cast<const uint8_t*>(blob),
                               static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
-                              static_cast<uint8_t*>(workspace));
+                              p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace));
+}
+
+template <int BITS>
+static cudaError_t launch_bits(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K, int N,
+                               void* workspace, cudaStream_t stream) {
+    // the cluster instructions are compiled only into the instantiations that are launched as clusters
+    if (p.cluster > 1) {
+        if (M > 8) return launch_one<BITS, 2, true, true>(p, blob, a, y, M, K, N, workspace, stream);
+        return p.full ? launch_one<BITS, 1, true, true>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<BITS, 1, false, true>(p, blob, a, y, M, K, N, workspace, stream);
+    }
+    if (M > 8) return launch_one<BITS, 2, true, false>(p, blob, a, y, M, K, N, workspace, stream);
+    return p.full ? launch_one<BITS, 1, true, false>(p, blob, a, y, M, K, N, workspace, stream)
+                  : launch_one<BITS, 1, false, false>(p, blob, a, y, M, K, N, workspace, stream);
 }
 
 cudaError_t launch_gemv(int bits, const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                         int N, void* workspace, cudaStream_t stream) {
-    if (bits == 4) {
-        if (M > 8) return launch_one<4, 2, true>(p, blob, a, y, M, K, N, workspace, stream);
-        return p.full ? launch_one<4, 1, true>(p, blob, a, y, M, K, N, workspace, stream)
-                      : launch_one<4, 1, false>(p, blob, a, y, M, K, N, workspace, stream);
-    }
-    if (M > 8) return launch_one<8, 2, true>(p, blob, a, y, M, K, N, workspace, stream);
-    return p.full ? launch_one<8, 1, true>(p, blob, a, y, M, K, N, workspace, stream)
-                  : launch_one<8, 1, false>(p, blob, a, y, M, K, N, workspace, stream);
+    return bits == 4 ? launch_bits<4>(p, blob, a, y, M, K, N, workspace, stream)
+                     : launch_bits<8>(p, blob, a, y, M, K, N, workspace, stream);
 }
 
 }  // namespace tf

@@ -14,6 +14,7 @@ __host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return
 __host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
 constexpr int kGemvFullFromBytes = 384 * 1024; // packed bytes per CTA from which up to 8 tokens use the whole-SM configuration
+constexpr int kGemvMaxDevices = 64;            // devices the per-device caches cover
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
 constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
@@ -34,6 +35,9 @@ struct GemvPlan {
     int consumers;     // consumer warps
     int stages;        // ring depth
     bool full;         // whole-SM configuration
+    int cluster;       // CTAs per cluster (1 = global mode: cut strips go through the workspace)
+    int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster)
+    int xslot_bytes;   // cluster mode: bytes of one partial-sum slot in shared memory
     int stage_bytes;   // bytes of one ring stage (weights + activations)
     int smem_bytes;
     int strips, ktiles, total_tiles;
