@@ -523,31 +523,39 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     }
 }
 
-// How many clusters of `csize` whole-SM CTAs the device can hold at once (asked once per device; half-SM CTAs fit
-// at least as often).  0 if the question fails: cluster mode is then not used.
-static int max_resident_clusters(int csize) {
-    static int cached[kGemvMaxDevices][4];      // [device][log2 csize], 0 = not asked yet, -1 = failed
+// How many clusters of `csize` CTAs the device can hold at once, for half-SM CTAs (two per SM) or whole-SM ones
+// (asked once per device).  0 if the question fails: cluster mode is then not used.
+static int max_resident_clusters(int csize, bool full) {
+    static int cached[kGemvMaxDevices][2][4];   // [device][full][log2 csize], 0 = not asked yet, -1 = failed
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kGemvMaxDevices) return 0;
     const int slot = csize == 2 ? 1 : csize == 4 ? 2 : 3;
-    if (cached[dev][slot] == 0) {
+    int& entry = cached[dev][full ? 1 : 0][slot];
+    if (entry == 0) {
         int n = 0;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(csize * 32, 1, 1);
-        cfg.blockDim = dim3(gemv_max_threads(1, true), 1, 1);
-        cfg.dynamicSmemBytes = gemv_smem_budget(1, true);
+        cfg.gridDim = dim3(csize * 64, 1, 1);
+        cfg.blockDim = dim3(gemv_max_threads(1, full), 1, 1);
+        cfg.dynamicSmemBytes = gemv_smem_budget(1, full);
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             gemv_smem_budget(1, true));
-        if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, true, true>, &cfg);
+        cudaError_t e;
+        if (full) {
+            e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gemv_smem_budget(1, true));
+            if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, true, true>, &cfg);
+        } else {
+            e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gemv_smem_budget(1, false));
+            if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, false, true>, &cfg);
+        }
         if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
-        cached[dev][slot] = n > 0 ? n : -1;
+        entry = n > 0 ? n : -1;
     }
-    return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
+    return entry > 0 ? entry : 0;
 }
 
 // Launch geometry.  Global mode: one persistent CTA per SM (fewer when there are fewer tiles than SMs), all tiles
@@ -570,8 +578,10 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.nclusters = 0;
     int best_t = 0;
     for (int c = 2; c <= 8; c *= 2) {
-        int maxc = max_resident_clusters(c);
-        if (maxc > sm_count / c) maxc = sm_count / c;
+        // up to 8 tokens a cluster-mode CTA is always a half-SM one (short ranges), so two fit on an SM
+        int maxc = max_resident_clusters(c, mt == 2);
+        const int slots = (mt == 2 ? 1 : 2) * sm_count / c;
+        if (maxc > slots) maxc = slots;
         if (maxc < 1) continue;
         const int j = (p.strips + maxc - 1) / maxc;                 // whole strips per cluster, at most
         const int ncl = (p.strips + j - 1) / j;
