@@ -578,10 +578,10 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.nclusters = 0;
     int best_t = 0;
     for (int c = 2; c <= 8; c *= 2) {
-        // up to 8 tokens a cluster-mode CTA is always a half-SM one (short ranges), so two fit on an SM
+        // one CTA per SM even where two half-SM ones would fit: the other half is where the next GEMV's CTAs
+        // wait with their rings full (measured: filling both halves shortens the call and lengthens the step)
         int maxc = max_resident_clusters(c, mt == 2);
-        const int slots = (mt == 2 ? 1 : 2) * sm_count / c;
-        if (maxc > slots) maxc = slots;
+        if (maxc > sm_count / c) maxc = sm_count / c;
         if (maxc < 1) continue;
         const int j = (p.strips + maxc - 1) / maxc;                 // whole strips per cluster, at most
         const int ncl = (p.strips + j - 1) / j;
