@@ -591,7 +591,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     // worth it for short ranges only (there the hand-over dominates the call), and only if the longest range stays
     // within one round of the consumer warps or close to the evenly split one
     const int one_round = gemv_max_consumers(mt, mt == 2);
-    if (p.cluster > 1 && tiles_per_cta <= 32 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
+    if (p.cluster > 1 && tiles_per_cta <= 16 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
         p.grid = p.nclusters * p.cluster;
         tiles_per_cta = best_t;
     } else {
