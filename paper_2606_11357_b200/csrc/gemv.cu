@@ -588,10 +588,13 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
         const int t = (j * p.ktiles + c - 1) / c;                   // longest range of a CTA
         if (p.cluster == 1 || t < best_t) { p.cluster = c; p.nclusters = ncl; best_t = t; }
     }
-    // worth it for short ranges only (there the hand-over dominates the call), and only if the longest range stays
-    // within one round of the consumer warps or close to the evenly split one
+    // Worth it for short ranges only (there the hand-over dominates the call), only if the longest range stays
+    // within one round of the consumer warps or close to the evenly split one, and only for the whole-SM
+    // configuration of 9..16 tokens: a half-SM GEMV overlaps its start with the previous kernel's end, a cluster
+    // launch next to a plain one does not (about 2.7 us per transition, measured), and in a pass over layers of
+    // different sizes that loss is larger than what the short hand-over wins for up to 8 tokens.
     const int one_round = gemv_max_consumers(mt, mt == 2);
-    if (p.cluster > 1 && tiles_per_cta <= 16 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
+    if (p.cluster > 1 && mt == 2 && tiles_per_cta <= 16 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
         p.grid = p.nclusters * p.cluster;
         tiles_per_cta = best_t;
     } else {
