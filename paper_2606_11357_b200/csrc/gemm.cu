@@ -125,7 +125,7 @@ __device__ __forceinline__ uint32_t bf16_dup(float v) {
 template <int BITS, int BT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
-            __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int n_tiles, int m_tiles,
+            __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int n_tiles, int m_tiles, int aligned,
             uint8_t* __restrict__ workspace) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
@@ -145,8 +145,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_units = n_tiles * m_tiles * ktiles;   // unit = (output tile, k-tile of 128)
-    const int u_begin = unit_start(blockIdx.x, total_units, gridDim.x);
-    const int u_end = unit_start(blockIdx.x + 1, total_units, gridDim.x);
+    // aligned: whole tiles only (no tile is shared between CTAs); otherwise the units are split evenly
+    const int total_tiles = n_tiles * m_tiles;
+    const int u_begin = aligned ? unit_start(blockIdx.x, total_tiles, gridDim.x) * ktiles : unit_start(blockIdx.x, total_units, gridDim.x);
+    const int u_end = aligned ? unit_start(blockIdx.x + 1, total_tiles, gridDim.x) * ktiles : unit_start(blockIdx.x + 1, total_units, gridDim.x);
     const Segments segs(u_begin, u_end, ktiles);
     const int strips = (N + kTileN - 1) / kTileN;
     const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N);
@@ -495,9 +497,20 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     const int n_tiles = (N + kBN - 1) / kBN, m_tiles = (M + BT - 1) / BT;
     const long long units = (long long)n_tiles * m_tiles * (K / kTileK);
     if (sm_count > kGemmMaxGrid) sm_count = kGemmMaxGrid;
-    const int grid = units < sm_count ? (int)units : sm_count;
+    // Two ways to spread the work.  Even split of the (tile, k-tile) units: no SM idles, but a CTA whose range
+    // holds no whole tile finishes with the fix-up of a cut tile in the open (about 18 k-tile times for a
+    // 256-token tile, measured; less for narrower tiles).  Whole tiles only: no fix-up, but the last wave of
+    // tiles may leave SMs idle.  Take the cheaper one, in k-tile times of the longest CTA.
+    const int ktiles = K / kTileK, tiles = n_tiles * m_tiles;
+    int grid = units < sm_count ? (int)units : sm_count;
+    const long long split_len = (units + grid - 1) / grid;
+    const long long split_cost = split_len + (split_len < 2 * ktiles ? 18 * BT / 256 : 0);
+    const int tile_grid = tiles < sm_count ? tiles : sm_count;
+    const long long tile_cost = (long long)((tiles + tile_grid - 1) / tile_grid) * ktiles;
+    const int aligned = tile_cost <= split_cost ? 1 : 0;
+    if (aligned) grid = tile_grid;
     gemm_kernel<BITS, BT><<<grid, kGemmThreads, gemm_smem_bytes(BITS, BT), stream>>>(
-        map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K, N, K / kTileK, n_tiles, m_tiles,
+        map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K, N, ktiles, n_tiles, m_tiles, aligned,
         static_cast<uint8_t*>(workspace));
     return cudaGetLastError();
 }
