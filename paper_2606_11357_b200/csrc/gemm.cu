@@ -113,6 +113,7 @@ struct GemmBarriers {
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t last_flag;
+    uint32_t deferred_tile;     // 1 + the cut tile this CTA finishes with all its warps after the role loops (0 = none)
 };
 
 __device__ __forceinline__ uint32_t bf16_dup(float v) {
@@ -170,6 +171,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
         mbar_init(smem_u32(&bars->acc_full), 1);
         mbar_init(smem_u32(&bars->acc_empty), 4);            // four epilogue warps
         bars->abort_flag = 0;
+        bars->deferred_tile = 0;
         mbar_init_fence();
     }
     if (warp == 2) {
@@ -409,7 +411,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                         bars->last_flag = (prev == (uint32_t)(ncontrib - 1)) ? 1u : 0u;
                     }
                     asm volatile("bar.sync 2, 128;" ::: "memory");
-                    if (*reinterpret_cast<volatile uint32_t*>(&bars->last_flag) != 0) {
+                    if (*reinterpret_cast<volatile uint32_t*>(&bars->last_flag) != 0 && seg_it + 1 == (uint32_t)segs.count) {
+                        // nothing left to hide the fix-up behind: every warp of the CTA takes a share of it after the
+                        // role loops (four warps alone are bound by the latency of their few loads in flight)
+                        if (warp == 12 && lane == 0) bars->deferred_tile = (uint32_t)tile + 1u;
+                    } else if (*reinterpret_cast<volatile uint32_t*>(&bars->last_flag) != 0) {
                         // sum in CTA order whoever arrived last; only the first contributor can hold a tail slot
                         const float4* first = reinterpret_cast<const float4*>(partials) +
                             (size_t)(c_first * 2 + (unit_start(c_first, total_units, gridDim.x) >= tile * ktiles ? 0 : 1)) * kSlotVec + row;
@@ -445,8 +451,64 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
         }
     }
 
-    // ---------------- teardown --------------------------------------------------------------------------------
+    // ---------------- deferred fix-up of the CTA's last cut tile, by all 16 warps --------------------------------
     tc_fence_before();
+    __syncthreads();
+    if (header_ok && bars->deferred_tile != 0 && bars->abort_flag == 0) {
+        // all MMAs of this CTA have completed, so the activation ring is free: one 1 KB transpose buffer per warp
+        const int tile = (int)bars->deferred_tile - 1;
+        const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
+        const int quarter = warp & 3, part = warp >> 2;               // rows 32 quarter .. +31, chunks part, part + 4, ..
+        const int row = 32 * quarter + lane;
+        __nv_bfloat16* tbuf = reinterpret_cast<__nv_bfloat16*>(act_ring + warp * kEpiWarpBytes);
+        constexpr size_t kSlotVec = (size_t)kBN * BT / 4;
+        const float4* partials4 = reinterpret_cast<const float4*>(workspace + kGemmPartialOffset);
+        const int c_first = unit_owner(tile * ktiles, total_units, gridDim.x);
+        const int ncontrib = unit_owner(tile * ktiles + ktiles - 1, total_units, gridDim.x) - c_first + 1;
+        const float4* first = partials4 +
+            (size_t)(c_first * 2 + (unit_start(c_first, total_units, gridDim.x) >= tile * ktiles ? 0 : 1)) * kSlotVec + row;
+        const float4* rest = partials4 + (size_t)((c_first + 1) * 2) * kSlotVec + row;     // later contributors: head slots
+        const int n8 = n_tile * kBN + 32 * quarter + 8 * (lane & 3);
+#pragma unroll 1
+        for (int c = part; c < BT / 16; c += 4) {
+            float4 acc4[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc4[j] = __ldcg(first + (4 * c + j) * kBN);
+            for (int cc = 1; cc < ncontrib; cc += 2) {                 // CTA order; two contributors' loads in flight
+                float4 x[4], z[4];
+                const float4* s0 = rest + (size_t)(cc - 1) * 2 * kSlotVec;
+                const bool two = cc + 1 < ncontrib;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) x[j] = __ldcg(s0 + (4 * c + j) * kBN);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) z[j] = two ? __ldcg(s0 + 2 * kSlotVec + (4 * c + j) * kBN) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc4[j].x += x[j].x; acc4[j].y += x[j].y; acc4[j].z += x[j].z; acc4[j].w += x[j].w;
+                    if (two) { acc4[j].x += z[j].x; acc4[j].y += z[j].y; acc4[j].z += z[j].z; acc4[j].w += z[j].w; }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                tbuf[(4 * j + 0) * 32 + lane] = __float2bfloat16_rn(acc4[j].x);
+                tbuf[(4 * j + 1) * 32 + lane] = __float2bfloat16_rn(acc4[j].y);
+                tbuf[(4 * j + 2) * 32 + lane] = __float2bfloat16_rn(acc4[j].z);
+                tbuf[(4 * j + 3) * 32 + lane] = __float2bfloat16_rn(acc4[j].w);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int tl = 8 * i + (lane >> 2);
+                const int tok = m_tile * BT + 16 * c + tl;
+                const uint4 d = *reinterpret_cast<const uint4*>(tbuf + tl * 32 + 8 * (lane & 3));
+                if (tok < M && n8 < N) *reinterpret_cast<uint4*>(y + (size_t)tok * N + n8) = d;
+            }
+            __syncwarp();
+        }
+        if (threadIdx.x == 0) reinterpret_cast<uint32_t*>(workspace + kGemmCounterOffset)[tile] = 0;   // ready for the next call
+    }
+
+    // ---------------- teardown --------------------------------------------------------------------------------
     __syncthreads();
     if (threadIdx.x == 0) {
         if (!header_ok) {
@@ -498,13 +560,13 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     const long long units = (long long)n_tiles * m_tiles * (K / kTileK);
     if (sm_count > kGemmMaxGrid) sm_count = kGemmMaxGrid;
     // Two ways to spread the work.  Even split of the (tile, k-tile) units: no SM idles, but a CTA whose range
-    // holds no whole tile finishes with the fix-up of a cut tile in the open (about 18 k-tile times for a
+    // holds no whole tile finishes with the fix-up of a cut tile in the open (about 10 k-tile times for a
     // 256-token tile, measured; less for narrower tiles).  Whole tiles only: no fix-up, but the last wave of
     // tiles may leave SMs idle.  Take the cheaper one, in k-tile times of the longest CTA.
     const int ktiles = K / kTileK, tiles = n_tiles * m_tiles;
     int grid = units < sm_count ? (int)units : sm_count;
     const long long split_len = (units + grid - 1) / grid;
-    const long long split_cost = split_len + (split_len < 2 * ktiles ? 18 * BT / 256 : 0);
+    const long long split_cost = split_len + (split_len < 2 * ktiles ? 10 * BT / 256 : 0);
     const int tile_grid = tiles < sm_count ? tiles : sm_count;
     const long long tile_cost = (long long)((tiles + tile_grid - 1) / tile_grid) * ktiles;
     const int aligned = tile_cost <= split_cost ? 1 : 0;
