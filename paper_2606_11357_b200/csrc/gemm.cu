@@ -56,9 +56,10 @@ __host__ __device__ constexpr int act_stages(int bits, int bt) {
                : (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt);
 }
 constexpr int kEpiWarpBytes = 1024;       // per epilogue warp: 16 tokens x 32 columns of bf16, for the transpose
+constexpr int kDrainWarpBytes = 512;      // per dequant warp: 8 tokens x 32 columns, for its share of an accumulator drain
 __host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
     return 1024 /*alignment slack*/ + act_stages(bits, bt) * act_stage_bytes(bt) +
-           kWpStages * 2 * wp_strip_bytes(bits) + 4 * kEpiWarpBytes + 512;
+           kWpStages * 2 * wp_strip_bytes(bits) + 4 * kEpiWarpBytes + 8 * kDrainWarpBytes + 512;
 }
 
 // workspace: [0,16) status | [kGemmCounterOffset, +4 * tiles) arrival counters | partial accumulators, two
@@ -116,6 +117,30 @@ struct GemmBarriers {
     uint32_t deferred_tile;     // 1 + the cut tile this CTA finishes with all its warps after the role loops (0 = none)
 };
 
+// One warp's share of the drain of a whole 128 x BT accumulator: the 8-token chunks `part`, `part + 3`, ... of its
+// lane quarter.  TMEM -> bf16 -> transposed through a 512-byte buffer -> one 16-byte store per lane (8 weight
+// columns of one token).  Three warps per quarter (one epilogue warp, two dequant warps) share a tile.
+template <int BT>
+__device__ __forceinline__ void drain_share(uint32_t tmem_base, __nv_bfloat16* tbuf8, __nv_bfloat16* y, int M, int N, int n_tile,
+                                            int m_tile, int quarter, int part, int lane) {
+    const uint32_t taddr = tmem_base + (uint32_t(32 * quarter) << 16);
+    const int n8 = n_tile * 128 + 32 * quarter + 8 * (lane & 3);
+    const int tl = lane >> 2;
+#pragma unroll 1
+    for (int c = part; c < BT / 8; c += 3) {
+        uint32_t r[8];
+        tmem_ld_32x32b_x8(taddr + 8 * c, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) tbuf8[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(r[j]));
+        __syncwarp();
+        const int tok = m_tile * BT + 8 * c + tl;
+        const uint4 d = *reinterpret_cast<const uint4*>(tbuf8 + tl * 32 + 8 * (lane & 3));
+        if (tok < M && n8 < N) *reinterpret_cast<uint4*>(y + (size_t)tok * N + n8) = d;
+        __syncwarp();
+    }
+}
+
 __device__ __forceinline__ uint32_t bf16_dup(float v) {
     const uint32_t b = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
     return b | (b << 16);
@@ -141,7 +166,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     uint8_t* act_ring = smem;                                        // kStages x kActStage   (1024-aligned)
     uint8_t* wp_ring = act_ring + kStages * kActStage;               // kWpStages x packed tiles
     uint8_t* epi_buf = wp_ring + kWpStages * kWpStageBytes;          // 4 x kEpiWarpBytes
-    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(epi_buf + 4 * kEpiWarpBytes);
+    uint8_t* drain_buf = epi_buf + 4 * kEpiWarpBytes;                // 8 x kDrainWarpBytes
+    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(drain_buf + 8 * kDrainWarpBytes);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -169,7 +195,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             mbar_init(smem_u32(&bars->wp_empty[s]), 8);      // all eight dequant warps
         }
         mbar_init(smem_u32(&bars->acc_full), 1);
-        mbar_init(smem_u32(&bars->acc_empty), 4);            // four epilogue warps
+        mbar_init(smem_u32(&bars->acc_empty), 12);           // four epilogue warps + eight dequant warps (drain duty)
         bars->abort_flag = 0;
         bars->deferred_tile = 0;
         mbar_init_fence();
@@ -260,12 +286,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             const int g = lane >> 2;
             uint32_t wit = 0;
             bool ok = true;
+            // Drain duty: every segment's accumulator is released by twelve arrivals, the four epilogue warps and
+            // these eight.  For a whole tile a dequant warp first drains its third of its lane quarter.  The duty
+            // for segment s is done just before this warp's third job after the end of s: the first job whose
+            // operand stage can only be freed by an MMA of segment s + 1, which in turn waits for that release.
+            int duty = 0;
+            __nv_bfloat16* tbuf8 = reinterpret_cast<__nv_bfloat16*>(drain_buf + (warp - 4) * kDrainWarpBytes);
+            auto do_duty = [&](int sidx) -> bool {
+                int dtile, dkt0, dlen, dslot;
+                segs.get(sidx, dtile, dkt0, dlen, dslot);
+                if (!mbar_wait(smem_u32(&bars->acc_full), sidx & 1, abort_flag, 0x520)) return false;
+                tc_fence_after();
+                if (dslot < 0) {
+                    const int dn = dtile / m_tiles, dm = dtile - dn * m_tiles;
+                    drain_share<BT>(tmem_base, tbuf8, y, M, N, dn, dm, q, 1 + half, lane);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty));
+                return true;
+            };
             for (int i = 0; i < segs.count && ok; ++i) {
                 int tile, kt0, len, slot;
                 segs.get(i, tile, kt0, len, slot);
                 const int n_tile = tile / m_tiles;
                 const bool strip_exists = 2 * n_tile + strip_sel < strips;
                 for (int T = kt0; T < kt0 + len; ++T, ++wit) {
+                    while (ok && (duty < i - 1 || (duty < i && T - kt0 >= 2))) ok = do_duty(duty++);
+                    if (!ok) break;
                     const int ws = wit % kWpStages;
                     ok = mbar_wait(smem_u32(&bars->wp_full[ws]), (wit / kWpStages) & 1, abort_flag, 0x500 + ws);
                     if (!ok) break;
@@ -339,6 +387,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[sa]));
                 }
             }
+            while (ok && duty < segs.count) ok = do_duty(duty++);
         } else if (warp >= 12) {
             // ================= epilogue: TMEM -> bf16 -> y, or -> fp32 partial for a tile cut between CTAs ==========
             const int quarter = warp & 3;                     // this warp may touch TMEM lanes 32*quarter .. +31
@@ -371,17 +420,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 if (!mbar_wait(smem_u32(&bars->acc_full), seg_it & 1, abort_flag, 0x600)) break;
                 tc_fence_after();
                 if (slot < 0) {
-                    // ---- the whole K range of the tile was computed here: round and store ----------------------
-#pragma unroll 1
-                    for (int c = 0; c < BT / 16; ++c) {
-                        uint32_t r[16];
-                        float v[16];
-                        tmem_ld_32x32b_x16(taddr + 16 * c, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                        store_chunk(v, n_tile, m_tile, c);
-                    }
+                    // ---- the whole K range of the tile was computed here: round and store this warp's third ---------
+                    drain_share<BT>(tmem_base, tbuf, y, M, N, n_tile, m_tile, quarter, 0, lane);
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty));
