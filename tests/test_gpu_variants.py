@@ -53,3 +53,23 @@ def test_illegal_group_sizes_are_rejected():
     assert tf.tf_packed_size(4, 1024, 64, 64) == 0          # below the tile's k-extent
     assert tf.tf_packed_size(4, 1024, 64, 384) == 0         # does not divide K
     assert tf.tf_packed_size(8, 1024, 64, 1024) > 0
+
+
+@pytest.mark.parametrize("kind,M,K,N,zero_bytes", [("gemv", 1, 4096, 1024, 4096), ("gemv", 16, 4096, 4096, 4096),
+                                                   ("gemv", 4, 1536, 328, 4096), ("gemm", 300, 2048, 1096, 20480),
+                                                   ("gemm", 512, 4096, 640, 20480)])
+def test_workspace_head_is_left_zero(kind, M, K, N, zero_bytes):
+    """The status word and the arrival counters must be zero again after a call, so the same workspace serves
+    the next call without being cleared."""
+    p = wl.make_w4(M, K, N, seed=900 + M)
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    a = gu.to_device_bf16(p.a_bf16)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    op = tf.TF_OP_GEMV_W4A16 if kind == "gemv" else tf.TF_OP_GEMM_W4A16
+    ws = torch.zeros(tf.tf_workspace_size(op, M, K, N), dtype=torch.uint8, device="cuda")
+    fn = tf.tf_gemv_w4a16 if kind == "gemv" else tf.tf_gemm_w4a16
+    for _ in range(3):
+        fn(blob, a, y, M, K, N, ws)
+    assert tf.tf_device_status(ws) == 0
+    assert int(ws[:zero_bytes].to(torch.int32).sum().item()) == 0
+    gu.check_against_oracle(p, gu.bits_of(y))
