@@ -134,14 +134,17 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     // "Contributor space": the CTAs that split one pool of tiles evenly among themselves.  Global mode: all CTAs
     // of the grid over all tiles.  Cluster mode: the CTAs of one cluster over the whole strips that cluster owns,
     // so that a strip is only ever shared inside a cluster and can be summed through distributed shared memory.
-    int cn = gridDim.x, crank = cta, cbase = 0, ctiles = total_tiles;
+    // In global mode `nclusters` carries the number of CTAs that take part (the first ones of the grid); the rest
+    // of the grid has no tiles and only keeps one CTA of this kernel on every SM (see plan_gemv).
+    int cn = nclusters, crank = cta, cbase = 0, ctiles = total_tiles;
     if (CL && csize > 1) {
         const int q = cta / csize, strips = total_tiles / ktiles;
         const int s0 = (int)(((long long)q * strips) / nclusters), s1 = (int)(((long long)(q + 1) * strips) / nclusters);
         cn = csize; crank = cta - q * csize; cbase = s0 * ktiles; ctiles = (s1 - s0) * ktiles;
     }
-    const int t0 = cbase + range_start(crank, ctiles, cn);
-    const int ntiles = cbase + range_start(crank + 1, ctiles, cn) - t0;
+    const bool idle = crank >= cn;
+    const int t0 = idle ? 0 : cbase + range_start(crank, ctiles, cn);
+    const int ntiles = idle ? 0 : cbase + range_start(crank + 1, ctiles, cn) - t0;
     int fin_strip = -1, fin_first = 0;          // cluster mode: the strip this CTA finishes after the cluster barrier
 
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
@@ -574,6 +577,30 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.grid = p.total_tiles < sm_count ? p.total_tiles : sm_count;
     const int mt = M <= 8 ? 1 : 2;
     int tiles_per_cta = (p.total_tiles + p.grid - 1) / p.grid;
+    // CTAs that get tiles.  The grid of a half-SM launch stays at one CTA per SM even when fewer take part: the
+    // block scheduler puts the next GEMV's CTAs wherever a half SM is free, and an SM without a CTA of this
+    // kernel would get two of them, which then share one SM for their whole range (measured: 2.5 us per call).
+    int active = p.grid;
+    // Short ranges (at most two rounds of a half-SM CTA's consumer warps): the hand-over of cut strips is most of the
+    // call, so pick ranges that line up with the strips.  (a) Few tiles: no more CTAs than give every consumer warp
+    // one tile; the call lasts one tile-time either way, and a strip is shared by fewer CTAs.  (b) Otherwise a
+    // range length that divides a strip (or is a multiple of it) and needs no more rounds: every CTA then has one
+    // cut instead of two.
+    if (mt == 1) {
+        const int nc = gemv_max_consumers(1, false);
+        int want = 0;
+        if (tiles_per_cta < nc) {
+            want = nc;
+        } else if (tiles_per_cta <= 2 * nc) {
+            const int rounds = (tiles_per_cta + nc - 1) / nc;
+            for (int t = tiles_per_cta; t <= rounds * nc; ++t)
+                if ((p.ktiles % t == 0 || t % p.ktiles == 0) && p.total_tiles % t == 0) { want = t; break; }
+        }
+        if (want > 0) {
+            int g = (p.total_tiles + want - 1) / want;
+            if (g >= 1 && g < p.grid) { active = g; tiles_per_cta = (p.total_tiles + active - 1) / active; }
+        }
+    }
     p.cluster = 1;
     p.nclusters = 0;
     int best_t = 0;
@@ -599,7 +626,8 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
         tiles_per_cta = best_t;
     } else {
         p.cluster = 1;
-        p.nclusters = 0;
+        p.nclusters = active;
+        if (mt == 1 && p.grid < sm_count) p.grid = sm_count;
     }
     // Long ranges amortise the start of the kernel: take the whole SM (more consumer warps, deeper ring).  Short
     // ones gain more from the next GEMV's CTAs sitting beside this one's with their rings already full.

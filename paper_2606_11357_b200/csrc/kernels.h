@@ -36,7 +36,7 @@ struct GemvPlan {
     int stages;        // ring depth
     bool full;         // whole-SM configuration
     int cluster;       // CTAs per cluster (1 = global mode: cut strips go through the workspace)
-    int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster)
+    int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster); global mode: CTAs that get tiles
     int xslot_bytes;   // cluster mode: bytes of one partial-sum slot in shared memory
     int stage_bytes;   // bytes of one ring stage (weights + activations)
     int smem_bytes;
