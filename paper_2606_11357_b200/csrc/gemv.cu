@@ -510,6 +510,15 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         }
     }
 
+    // A CTA without tiles leaves about a microsecond after the dependency is met, not at once.  Measured: when the
+    // surplus CTAs of a short GEMV all exit in the instant the previous kernel completes, the kernels behind it
+    // on the stream are placed unevenly and a pass over four layer shapes takes 46 us instead of 37; any delay
+    // between 1 and 4 us gives the 37 (the CTAs with tiles need 3 us or more from that instant anyway).
+    if (idle && threadIdx.x == 0) {
+        const long long t_begin = clock64();
+        while (clock64() - t_begin < 2000ll) {}
+    }
+
     // ---------------- teardown: report, and never leave with copies in flight ------------------------------
     if (threadIdx.x == 0 && (!header_ok || *abort_flag != 0)) {
         grid_dependency_wait();
