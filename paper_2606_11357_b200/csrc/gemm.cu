@@ -589,7 +589,14 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     cudaError_t me = encode_bf16_map(&map, a, 2, dims, strides, box);
     if (me != cudaSuccess) return me;
 
-    static bool configured = false;
+    // function attributes belong to one device: set them once per device and kernel (twice is harmless)
+    constexpr int kMaxDevices = 64;
+    static bool configured_on[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    bool unseen = dev < 0 || dev >= kMaxDevices;
+    bool& configured = unseen ? unseen : configured_on[dev];
+    if (unseen) configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BITS, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              gemm_smem_bytes(BITS, BT));

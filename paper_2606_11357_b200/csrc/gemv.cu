@@ -672,7 +672,13 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     const cuuint32_t box[3] = {64, (cuuint32_t)(2 * gemv_chunk_tiles(BITS)), (cuuint32_t)M};
     cudaError_t me = encode_bf16_map(&map, a, 3, dims, strides, box);
     if (me != cudaSuccess) return me;
-    static bool configured = false;       // the attribute is per kernel; setting it twice is harmless
+    // function attributes belong to one device: set them once per device and kernel (twice is harmless)
+    static bool configured_on[kGemvMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    bool unseen = dev < 0 || dev >= kGemvMaxDevices;
+    bool& configured = unseen ? unseen : configured_on[dev];
+    if (unseen) configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              gemv_smem_budget(MT, FULL));
