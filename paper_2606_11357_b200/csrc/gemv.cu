@@ -47,6 +47,24 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
     return v;
 }
 
+// Integer warp MMA: D(16x8, s32) += A(16x32, s8) . B(32x8, s8).  Thread (g, t): a0 = row g, k 4t..4t+3; a1 = row g+8;
+// a2, a3 = the same rows, k + 16; b0 = column g, k 4t..4t+3; b1 = k + 16; d = rows g, g+8 x columns 2t, 2t+1.
+__device__ __forceinline__ void mma_s8_16832(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// The same with D = A . B (no accumulator to clear first).
+__device__ __forceinline__ void mma_s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    const int zero = 0;
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
+}
+
+// int -> float for |v| < 2^22 without the conversion unit: 1.5 * 2^23 + v is exact in fp32.
+__device__ __forceinline__ float small_int_to_float(int v) {
+    return __int_as_float(0x4B400000 + v) - 12582912.0f;
+}
+
 __device__ __forceinline__ int range_start(int cta, int total, int grid) {
     return static_cast<int>((static_cast<long long>(cta) * total) / grid);
 }
@@ -100,7 +118,7 @@ __device__ __forceinline__ void store_strip(__nv_bfloat16* y, const float4 (&tot
 
 }  // namespace
 
-template <int BITS, int MT, bool FULL, bool CL>
+template <int BITS, int MT, bool FULL, bool CL, bool I8>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
                    __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
@@ -127,7 +145,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
     // xred [csize][xslot]: in cluster mode, the partials other CTAs of the cluster send to the finisher of a strip
     uint8_t* xred = smem + kGemvBarrierBytes + nconsumers * kRedWarp * 4;
-    uint8_t* ring = xred + ((CL && csize > 1 ? csize * xslot_bytes : 0) + 1023) / 1024 * 1024;
+    // pscr [consumers][1 KB]: integer path, a warp's activation pieces of the tile it works on
+    uint32_t* pscr = reinterpret_cast<uint32_t*>(xred + ((CL && csize > 1 ? csize * xslot_bytes : 0) + 1023) / 1024 * 1024);
+    uint8_t* ring = reinterpret_cast<uint8_t*>(pscr) + (I8 ? nconsumers * 1024 : 0);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
@@ -394,6 +414,111 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     }
 
                 const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
+                if constexpr (I8) {
+                    // ---- integer path (int8 weights, 1 or 2 tokens): codes x activation pieces on the integer warp MMA ----
+                    // The 128 activations of a (token, k-tile) are scaled by 2^(148 - emax) (emax = largest biased
+                    // exponent among them), rounded to integers |v| < 2^22 and split into signed bytes
+                    // v = p0 + 256 p1 + 65536 p2: values within 2^14 of the largest are exact, smaller ones are rounded
+                    // at 2^-22 of it.  Piece j of token m is column 3m + j of the MMA's 8-column operand; the int8 codes
+                    // are the other operand as they are, so no weight is ever converted:
+                    //     D[n][3m+j] = sum_k q[k][n] p_j[m][k]            (exact, 32-bit integers)
+                    //     y[m][n] += s[n] 2^(emax-148) sum_j 256^j D[n][3m+j]
+                    static_assert(!I8 || (BITS == 8 && MT == 1), "the integer path is built for int8 weights and up to 2 tokens");
+                    uint32_t* scr = pscr + cw * 256;                    // [column][36 words]: word of lane L at (L&3)*8 + (L>>2)
+                    // [column]: 2^(emax-148) 256^j in 8-byte entries behind the 6 x 36 words, a thread's two columns = one 16-byte load
+                    // (with 4-byte entries and an 8-byte load the same kernel ran 12 % slower: measured, cause not established)
+                    uint2* col_meta = reinterpret_cast<uint2*>(scr + 216);
+#pragma unroll
+                    for (int m = 0; m < 2; ++m) {
+                        if (m < M) {
+                            // lane L holds k = 4L .. 4L+3 of the tile
+                            const int row = m * (2 * kR) + 2 * slot + (lane >> 4);
+                            const uint2 raw = lds_v2(smem_u32(stage + kActOffset) + row * 128 +
+                                                     (((((lane & 15) >> 1) ^ (row & 7))) << 4) + (lane & 1) * 8);
+                            const uint32_t x0 = raw.x, x1 = raw.y;
+                            uint32_t e = max(max((x0 << 17) >> 24, (x0 << 1) >> 24), max((x1 << 17) >> 24, (x1 << 1) >> 24));
+                            e = __reduce_max_sync(0xFFFFFFFFu, e);
+                            e = max(e, 22u);                                  // keeps both powers of two normal numbers
+                            const float mult = __uint_as_float((275u - e) << 23);          // 2^(148 - emax)
+                            // v + 0x808080 has the bytes p0 + 128, p1 + 128, p2 + 128 of the balanced split
+                            uint32_t v[4];
+                            v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
+                            v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
+                            v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
+                            v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
+                            // 4 x 3 byte transpose: one word per piece, bytes in k order
+                            const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
+                            const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
+                            uint32_t word[3];
+                            word[0] = __byte_perm(ab01, cd01, 0x5410) ^ 0x80808080u;
+                            word[1] = __byte_perm(ab01, cd01, 0x7632) ^ 0x80808080u;
+                            word[2] = __byte_perm(ab2, cd2, 0x5410) ^ 0x80808080u;
+                            const float se = __uint_as_float((e - 21u) << 23);             // 2^(emax - 148)
+#pragma unroll
+                            for (int j = 0; j < 3; ++j) {
+                                const int c = 3 * m + j;
+                                scr[c * 36 + (lane & 3) * 8 + (lane >> 2)] = word[j];
+                                if (lane == 0) col_meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), 0u);
+                            }
+                        }
+                    }
+                    if (lane == 0) {                                    // columns without a token contribute nothing
+#pragma unroll
+                        for (int c = 3; c < 8; ++c)
+                            if (c >= 3 * M) col_meta[c] = make_uint2(0u, 0u);
+                    }
+                    __syncwarp();
+                    const uint4 cm = *reinterpret_cast<const uint4*>(col_meta + 2 * t);
+                    const float2 col_scale = make_float2(__uint_as_float(cm.x), __uint_as_float(cm.z));
+                    uint32_t bw[8];                                     // column g: the words of k-blocks 0..7 for this t
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) bw[i] = 0u;
+                    if (g < 3 * M) {
+                        const uint4 lo = *reinterpret_cast<const uint4*>(scr + g * 36 + t * 8);
+                        const uint4 hi = *reinterpret_cast<const uint4*>(scr + g * 36 + t * 8 + 4);
+                        bw[0] = lo.x; bw[1] = lo.y; bw[2] = lo.z; bw[3] = lo.w;
+                        bw[4] = hi.x; bw[5] = hi.y; bw[6] = hi.z; bw[7] = hi.w;
+                    }
+                    __syncwarp();                                       // the scratch is rewritten for the next tile
+                    int d[4][4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {                       // 32 k per MMA: k-blocks 2i and 2i+1
+                        uint4 wv[2][2];
+#pragma unroll
+                        for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                wv[hb][h] = *reinterpret_cast<const uint4*>(tile + ((size_t)((2 * i + hb) * 2 + h) * 32 + lane) * 16);
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            uint32_t a[4];
+#pragma unroll
+                            for (int hb = 0; hb < 2; ++hb) {
+                                const uint4 v = wv[hb][w >> 1];
+                                const uint32_t w0 = (w & 1) ? v.z : v.x, w1 = (w & 1) ? v.w : v.y;
+                                a[2 * hb] = __byte_perm(w0, w1, 0x5410);         // row g,   k 0..3 of this thread
+                                a[2 * hb + 1] = __byte_perm(w0, w1, 0x7632);     // row g+8
+                            }
+                            if (i == 0) mma_s8_16832_first(d[w], a[0], a[1], a[2], a[3], bw[0], bw[1]);
+                            else mma_s8_16832(d[w], a[0], a[1], a[2], a[3], bw[2 * i], bw[2 * i + 1]);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int tiles_here = min(kR, seg_len - cl * kR);
+                        mbar_arrive_n(empty0 + 8 * s, slot == tiles_here - 1 ? (uint32_t)(kR - tiles_here + 1) : 1u);
+                    }
+                    const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float s_g = fp16_bits_to_float((uint16_t)(sw[w] & 0xFFFFu));
+                        const float s_g8 = fp16_bits_to_float((uint16_t)(sw[w] >> 16));
+                        acc[w][0][0] = fmaf(small_int_to_float(d[w][0]) * col_scale.x, s_g, acc[w][0][0]);
+                        acc[w][0][1] = fmaf(small_int_to_float(d[w][1]) * col_scale.y, s_g, acc[w][0][1]);
+                        acc[w][0][2] = fmaf(small_int_to_float(d[w][2]) * col_scale.x, s_g8, acc[w][0][2]);
+                        acc[w][0][3] = fmaf(small_int_to_float(d[w][3]) * col_scale.y, s_g8, acc[w][0][3]);
+                    }
+                } else {
                 uint32_t zg[4], zg8[4];
                 if (BITS == 4) {
                     const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile + kWeightBytes + kScaleBytes) + g);
@@ -461,12 +586,31 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                         acc[w][mt][3] = fmaf(s_g8, gacc[w][mt][3], acc[w][mt][3]);
                     }
                 }
+                }
             }
             if (aborted) break;
 
             // ---- drop this warp's partial of the segment for the reducer and move on ---------------------------
             if (!mbar_wait(seg_free0, (sidx & 1) ^ 1, abort_flag, 0x300)) { aborted = true; break; }   // previous segment read
             float* mine = red + (size_t)cw * kRedWarp;                          // [token][n]
+            if constexpr (I8) {
+                // columns 3m .. 3m+2 are the pieces of token m, already on a common scale: add them up across the four
+                // threads of a row (fixed order) and leave tokens 0, 1 where the bf16 path has them (t = 0)
+#pragma unroll
+                for (int w = 0; w < 4; ++w)
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        const float c0 = acc[w][0][2 * r], c1 = acc[w][0][2 * r + 1];
+                        float tok0 = t == 0 ? c0 + c1 : t == 1 ? c0 : 0.f;
+                        float tok1 = t == 1 ? c1 : t == 2 ? c0 + c1 : 0.f;
+                        tok0 += __shfl_xor_sync(0xFFFFFFFFu, tok0, 1);
+                        tok1 += __shfl_xor_sync(0xFFFFFFFFu, tok1, 1);
+                        tok0 += __shfl_xor_sync(0xFFFFFFFFu, tok0, 2);
+                        tok1 += __shfl_xor_sync(0xFFFFFFFFu, tok1, 2);
+                        acc[w][0][2 * r] = t == 0 ? tok0 : 0.f;
+                        acc[w][0][2 * r + 1] = t == 0 ? tok1 : 0.f;
+                    }
+            }
 #pragma unroll
             for (int w = 0; w < 4; ++w)
 #pragma unroll
@@ -556,13 +700,13 @@ static int max_resident_clusters(int csize, bool full) {
         cfg.numAttrs = 1;
         cudaError_t e;
         if (full) {
-            e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gemv_smem_budget(1, true));
-            if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, true, true>, &cfg);
+            if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, true, true, false>, &cfg);
         } else {
-            e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(gemv_stream_kernel<4, 1, false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gemv_smem_budget(1, false));
-            if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, false, true>, &cfg);
+            if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, gemv_stream_kernel<4, 1, false, true, false>, &cfg);
         }
         if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
         entry = n > 0 ? n : -1;
@@ -649,8 +793,9 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
     // cluster mode: one slot per CTA of the cluster for the rows of real tokens (two token rows = 512 bytes)
     p.xslot_bytes = p.cluster > 1 ? ((M + 1) / 2) * 512 : 0;
+    p.i8 = bits == 8 && M <= kGemvI8MaxM && p.cluster == 1;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4 +
-                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024;
+                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (p.i8 ? p.consumers * 1024 : 0);
     int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
     if (stages > kGemvMaxStages) stages = kGemvMaxStages;
     // no more stages than the range has chunks
@@ -661,7 +806,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     return p;
 }
 
-template <int BITS, int MT, bool FULL, bool CL>
+template <int BITS, int MT, bool FULL, bool CL, bool I8>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
     // activations [M][K] seen as {64 k, K/64, M tokens} (strides increase with the dimension): one box = the
@@ -680,13 +825,13 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     bool& configured = unseen ? unseen : configured_on[dev];
     if (unseen) configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              gemv_smem_budget(MT, FULL));
         if (e != cudaSuccess) return e;
         // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
         // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
         // consecutive GEMVs of different shapes could not share an SM.
-        e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -709,7 +854,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
         attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
         cfg.numAttrs = 2;
     }
-    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL>, map, static_cast<const uint8_t*>(blob),
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8>, map, static_cast<const uint8_t*>(blob),
                               static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
                               p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace));
 }
@@ -719,13 +864,18 @@ static cudaError_t launch_bits(const GemvPlan& p, const void* blob, const void* 
                                void* workspace, cudaStream_t stream) {
     // the cluster instructions are compiled only into the instantiations that are launched as clusters
     if (p.cluster > 1) {
-        if (M > 8) return launch_one<BITS, 2, true, true>(p, blob, a, y, M, K, N, workspace, stream);
-        return p.full ? launch_one<BITS, 1, true, true>(p, blob, a, y, M, K, N, workspace, stream)
-                      : launch_one<BITS, 1, false, true>(p, blob, a, y, M, K, N, workspace, stream);
+        if (M > 8) return launch_one<BITS, 2, true, true, false>(p, blob, a, y, M, K, N, workspace, stream);
+        return p.full ? launch_one<BITS, 1, true, true, false>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<BITS, 1, false, true, false>(p, blob, a, y, M, K, N, workspace, stream);
     }
-    if (M > 8) return launch_one<BITS, 2, true, false>(p, blob, a, y, M, K, N, workspace, stream);
-    return p.full ? launch_one<BITS, 1, true, false>(p, blob, a, y, M, K, N, workspace, stream)
-                  : launch_one<BITS, 1, false, false>(p, blob, a, y, M, K, N, workspace, stream);
+    if (M > 8) return launch_one<BITS, 2, true, false, false>(p, blob, a, y, M, K, N, workspace, stream);
+    if constexpr (BITS == 8) {
+        if (p.i8)
+            return p.full ? launch_one<8, 1, true, false, true>(p, blob, a, y, M, K, N, workspace, stream)
+                          : launch_one<8, 1, false, false, true>(p, blob, a, y, M, K, N, workspace, stream);
+    }
+    return p.full ? launch_one<BITS, 1, true, false, false>(p, blob, a, y, M, K, N, workspace, stream)
+                  : launch_one<BITS, 1, false, false, false>(p, blob, a, y, M, K, N, workspace, stream);
 }
 
 cudaError_t launch_gemv(int bits, const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,

@@ -23,6 +23,7 @@ constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
 constexpr int kGemvActOffset = 17408;         // 17 x 1024 >= 4 x 4256 and >= 2 x 8320
 constexpr int kGemvMaxM = 16;
+constexpr int kGemvI8MaxM = 2;                // int8 weights, up to this many tokens: the GEMV runs on the integer warp MMA
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
 // Workspace layout: [0,16) status word | [256, 256+4*512) per-strip arrival counters | partial sums
 constexpr int kGemvCounterOffset = 256;
@@ -35,6 +36,7 @@ struct GemvPlan {
     int consumers;     // consumer warps
     int stages;        // ring depth
     bool full;         // whole-SM configuration
+    bool i8;           // integer path: int8 codes x activation pieces (W8, 1 or 2 tokens)
     int cluster;       // CTAs per cluster (1 = global mode: cut strips go through the workspace)
     int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster); global mode: CTAs that get tiles
     int xslot_bytes;   // cluster mode: bytes of one partial-sum slot in shared memory

@@ -73,3 +73,25 @@ def test_workspace_head_is_left_zero(kind, M, K, N, zero_bytes):
     assert tf.tf_device_status(ws) == 0
     assert int(ws[:zero_bytes].to(torch.int32).sum().item()) == 0
     gu.check_against_oracle(p, gu.bits_of(y))
+
+
+@pytest.mark.parametrize("M", [1, 2])
+@pytest.mark.parametrize("pattern", ["wide", "tiny_tile", "huge"])
+def test_w8_gemv_activation_dynamic_range(M, pattern):
+    """W8A16 with 1 or 2 tokens multiplies int8 codes with the activations of a k-tile written as integers on the
+    tile's own power-of-two scale; the result must stay inside the acceptance rule whatever the spread of magnitudes
+    inside a tile, from tile to tile, or the absolute magnitude."""
+    K, N = 2048, 328
+    p = wl.make_w8(M, K, N, seed=900 + M)
+    rng = np.random.default_rng(901 + M)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    if pattern == "wide":            # exponents spread over 40 binades inside every tile
+        a *= np.exp2(rng.integers(-30, 11, size=(M, K))).astype(np.float32)
+    elif pattern == "tiny_tile":     # whole k-tiles 2^-40 below their neighbours
+        a[:, 128:256] *= np.float32(2.0 ** -40)
+        a[:, 1024:1152] *= np.float32(2.0 ** -60)
+    else:                            # near the top and the bottom of the bf16 range
+        a[0] *= np.float32(2.0 ** 100)
+        a[M - 1, K // 2:] *= np.float32(2.0 ** -110)
+    p.a_bf16 = wl.f32_to_bf16_bits(a)
+    gu.check_against_oracle(p, gu.run(p, "gemv"))
