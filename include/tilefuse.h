@@ -150,6 +150,10 @@ tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s_fp16,
  *            workspace per stream: calls that run concurrently must not share one.
  * Arithmetic: weights are kept exact ((q - z) as small integers, scale applied in fp32 to
  * per-group partial sums), fp32 accumulation, one round-to-nearest-even to bf16 at the end.
+ * tf_gemv_w8a16 with M <= 2 forms the products in integers: per token and 128-deep k-tile the
+ * activations are rewritten on the tile's own power-of-two scale (exact for values within 2^14
+ * of the tile's largest magnitude, rounded at 2^-22 of it below that), multiplied with the int8
+ * codes exactly in 32 bits, and scaled back in fp32.
  * Each persistent CTA streams one contiguous range of packed tiles; a strip of 64 output
  * columns that is cut between CTAs is summed in CTA order by the last CTA to finish it.
  * The blob must be at least tf_packed_size(bits, K, N, 128) bytes for the K, N passed here.
