@@ -361,6 +361,50 @@ def run_gpu(args):
                                   "frac_of_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
                 del g, extra, blobs
 
+    # ---- one decoder layer at M = 1: seven GEMVs, or four after joining QKV and gate + up at pack time -------
+    decode_layer = None
+    if rank == 0:
+        def blob_of(K, N):
+            return next(c[4] for c in calls if (c[1], c[2], c[3]) == (1, K, N))
+        def act_of(K):
+            return next(c[5] for c in calls if c[1] == 1 and c[2] == K)
+        (Kh, Nh), (_, Nkv), (_, Nff), (Kff, _) = wl.LLAMA3_8B_SHAPES
+        bq, bkv, bff, bdown = blob_of(Kh, Nh), blob_of(Kh, Nkv), blob_of(Kh, Nff), blob_of(Kff, Nh)
+        host = lambda t: t.cpu().numpy()
+        bqkv = torch.from_numpy(tf.tf_pack_concat([host(bq), host(bkv), host(bkv)])).to(dev)
+        bgu = torch.from_numpy(tf.tf_pack_concat([host(bff), host(bff)])).to(dev)
+        a_h, a_ff = act_of(Kh), act_of(Kff)
+        y_big = torch.empty((1, 2 * Nff), dtype=torch.bfloat16, device=dev)
+        layers = {"unfused": [(bq, a_h, Kh, Nh), (bkv, a_h, Kh, Nkv), (bkv, a_h, Kh, Nkv), (bq, a_h, Kh, Nh),
+                              (bff, a_h, Kh, Nff), (bff, a_h, Kh, Nff), (bdown, a_ff, Kff, Nh)],
+                  "fused": [(bqkv, a_h, Kh, Nh + 2 * Nkv), (bq, a_h, Kh, Nh), (bgu, a_h, Kh, 2 * Nff), (bdown, a_ff, Kff, Nh)]}
+        decode_layer = {"M": 1, "note": "Llama-3-8B decoder layer, W4A16, CUDA graph of 3 layers on separate weight copies"}
+        for name, ops in layers.items():
+            copies = [[(b.clone(), a, K, N) for (b, a, K, N) in ops] for _ in range(3)]     # 3 x 113 MB > L2
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                for (b, a, K, N) in copies[0]:
+                    tf.tf_gemv_w4a16(b, a, y_big[:, :N], 1, K, N, ws, stream=stream)
+                stream.synchronize()
+                with torch.cuda.graph(g, stream=stream):
+                    for layer in copies:
+                        for (b, a, K, N) in layer:
+                            tf.tf_gemv_w4a16(b, a, y_big[:, :N], 1, K, N, ws, stream=stream)
+                g.replay()
+                stream.synchronize()
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0.record(stream)
+                for _ in range(10):
+                    g.replay()
+                s1.record(stream)
+                stream.synchronize()
+            decode_layer[name] = {"launches": len(ops), "us_per_layer": round(s0.elapsed_time(s1) * 1e3 / 30, 2)}
+            del g, copies
+        iso = {(r["K"], r["N"]): r["us"] for r in per_shape if r["M"] == 1}
+        decode_layer["sum_of_isolated_us"] = round(2 * iso[(Kh, Nh)] + 2 * iso[(Kh, Nkv)] + 2 * iso[(Kh, Nff)] + iso[(Kff, Nh)], 2)
+        assert tf.tf_device_status(ws) == 0
+        del bqkv, bgu
+
     # ---- prefill GEMM (config 2) ---------------------------------------------------------------------------
     gemm = None
     if rank == 0 and not args.skip_gemm:
@@ -450,6 +494,7 @@ def run_gpu(args):
                      "kernel": "gemv_stream_kernel (all 12 launches of the step)"},
         "cpu_baseline": cpu_baseline,
         "per_shape": per_shape,
+        "decode_layer": decode_layer,
         "gemm": gemm,
         "ceilings": ceilings,
     }

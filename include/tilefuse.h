@@ -138,6 +138,22 @@ tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s_fp16,
                        int K, int N, int group_size, void* cuda_stream);
 
 /*
+ * Concatenation along N at pack time.  Section 4.5: dispatching a kernel is amortized by a large
+ * prefill GEMM but costly for the short GEMV operators of token generation.  A decoder layer applies
+ * several weight matrices to the same activations; packing them side by side turns their GEMVs/GEMMs
+ * into one launch (fused QKV, fused gate + up).
+ *   parts    host, `count` pointers to blobs from tf_pack_awq / tf_pack_w8 (or from this call).
+ *   out      host, receives the blob of the matrix [W_0 | W_1 | ... ] with N = sum of the parts' N:
+ *            byte for byte what the packer gives for the column-concatenated inputs.
+ *   out_bytes  capacity of `out`; at least tf_packed_size(bits, K, N, group_size).
+ * All parts must have the same bits, K and group_size; every part but the last must have N % 64 == 0
+ * (it must end on a strip boundary); the total N must not exceed TF_MAX_DIM.  `out` must not overlap a part.
+ * Errors: TF_ERR_NULL, TF_ERR_BLOB (a part is not a valid blob), TF_ERR_SHAPE (count < 1, mismatch,
+ *         unaligned part, N too large), TF_ERR_WORKSPACE (out_bytes too small).
+ */
+tf_status tf_pack_concat(const void* const* parts, int count, void* out, size_t out_bytes);
+
+/*
  * Decode-phase fused GEMV (Sections 4.3 "GEMV microkernel" and 4.4): 1 <= M <= 16 tokens.
  *   packed   device, blob from tf_pack_awq (w4a16) / tf_pack_w8 (w8a16) for this K, N.
  *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.

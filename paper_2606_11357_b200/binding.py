@@ -20,7 +20,7 @@ TF_OP_GEMV_W4A16, TF_OP_GEMV_W8A16, TF_OP_GEMM_W4A16, TF_OP_GEMM_W8A16 = 0, 1, 2
 STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIGN", 4: "TF_ERR_BLOB",
                 5: "TF_ERR_WORKSPACE", 6: "TF_ERR_ARCH", 7: "TF_ERR_CUDA", 8: "TF_ERR_TIMEOUT"}
 
-EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_unpack_w4", "tf_unpack_w8",
+EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static")
 
@@ -45,6 +45,7 @@ def lib() -> ctypes.CDLL:
         L.tf_packed_size.restype, L.tf_packed_size.argtypes = c_size, [c_int] * 4
         L.tf_pack_awq.restype, L.tf_pack_awq.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, vp, c_size]
         L.tf_pack_w8.restype, L.tf_pack_w8.argtypes = c_int, [vp, vp, c_int, c_int, c_int, vp, c_size]
+        L.tf_pack_concat.restype, L.tf_pack_concat.argtypes = c_int, [vp, c_int, vp, c_size]
         L.tf_unpack_w4.restype, L.tf_unpack_w4.argtypes = c_int, [vp, vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_unpack_w8.restype, L.tf_unpack_w8.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, vp]
         for name in ("tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16"):
@@ -115,6 +116,17 @@ def tf_pack_w8(w_i8, scales_f16, K: int, N: int, group_size: int = 128, out=None
         out = np.empty(size, dtype=np.uint8)
     _check("tf_pack_w8", lib().tf_pack_w8(w.ctypes.data, scales.ctypes.data, K, N, group_size,
                                           out.ctypes.data, out.nbytes))
+    return out
+
+
+def tf_pack_concat(parts, out=None) -> np.ndarray:
+    """parts: packed blobs (uint8 numpy arrays) with the same bits, K and group size -> blob of [W_0 | W_1 | ...]."""
+    parts = [_host(p, np.uint8) for p in parts]
+    if out is None:
+        payload = sum(int(p.nbytes) - 256 for p in parts)
+        out = np.empty(256 + max(payload, 0), dtype=np.uint8)
+    ptrs = (ctypes.c_void_p * max(len(parts), 1))(*[p.ctypes.data for p in parts])
+    _check("tf_pack_concat", lib().tf_pack_concat(ctypes.cast(ptrs, ctypes.c_void_p), len(parts), out.ctypes.data, out.nbytes))
     return out
 
 

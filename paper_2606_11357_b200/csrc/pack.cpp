@@ -149,3 +149,40 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_pack_w8(const int
     }
     return TF_OK;
 }
+
+// Concatenation along N of blobs that share bits, K and group size (fused QKV, fused gate + up).  Section 4.5
+// names the cost of dispatching many short GEMV operators per token; fewer, wider operators is the remedy at pack time.  Tiles are stored strip after strip, so the tiles
+// of a part whose N is a multiple of the strip width are moved as they are; only the header changes.
+extern "C" __attribute__((visibility("default"))) tf_status tf_pack_concat(const void* const* parts, int count, void* out,
+                                                                           size_t out_bytes) {
+    if (!parts || !out) return TF_ERR_NULL;
+    if (count < 1) return TF_ERR_SHAPE;
+    tf_blob_header first;
+    long long n_total = 0;
+    for (int i = 0; i < count; ++i) {
+        if (!parts[i]) return TF_ERR_NULL;
+        tf_blob_header h;
+        memcpy(&h, parts[i], sizeof(h));
+        if (h.magic != tf::kMagic || h.version != tf::kBlobVersion) return TF_ERR_BLOB;
+        if (h.total_bytes != tf_packed_size((int)h.bits, (int)h.K, (int)h.N, (int)h.group_size) || h.total_bytes == 0)
+            return TF_ERR_BLOB;
+        if (i == 0) first = h;
+        else if (h.bits != first.bits || h.K != first.K || h.group_size != first.group_size) return TF_ERR_SHAPE;
+        if (i + 1 < count && h.N % tf::kTileN != 0) return TF_ERR_SHAPE;   // a part that is not last must end on a strip
+        n_total += h.N;
+    }
+    if (n_total > TF_MAX_DIM) return TF_ERR_SHAPE;
+    const size_t total = tf_packed_size((int)first.bits, (int)first.K, (int)n_total, (int)first.group_size);
+    if (total == 0) return TF_ERR_SHAPE;
+    if (out_bytes < total) return TF_ERR_WORKSPACE;
+    uint8_t* dst = static_cast<uint8_t*>(out) + tf::kHeaderBytes;
+    for (int i = 0; i < count; ++i) {
+        tf_blob_header h;
+        memcpy(&h, parts[i], sizeof(h));
+        const size_t payload = (size_t)h.total_bytes - tf::kHeaderBytes;
+        memcpy(dst, static_cast<const uint8_t*>(parts[i]) + tf::kHeaderBytes, payload);
+        dst += payload;
+    }
+    write_header(out, (int)first.bits, (int)first.K, (int)n_total, (int)first.group_size, total);
+    return TF_OK;
+}

@@ -95,3 +95,26 @@ def test_w8_gemv_activation_dynamic_range(M, pattern):
         a[M - 1, K // 2:] *= np.float32(2.0 ** -110)
     p.a_bf16 = wl.f32_to_bf16_bits(a)
     gu.check_against_oracle(p, gu.run(p, "gemv"))
+
+
+@pytest.mark.parametrize("kind,M", [("gemv", 1), ("gemv", 16), ("gemm", 200)])
+def test_fused_qkv_blob_from_pack_concat(kind, M):
+    """Three weight matrices packed separately, joined with tf_pack_concat, multiplied in one launch: the result
+    is the oracle's for the column-concatenated matrix (Section 4.5: fewer, wider operators per token)."""
+    K, widths = 1024, (512, 128, 128)
+    parts = [wl.make_w4(M, K, n, seed=800 + i) for i, n in enumerate(widths)]
+    for p in parts[1:]:
+        p.a_bf16 = parts[0].a_bf16
+    blobs = [tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, K, p.N) for p in parts]
+    whole = wl.Problem("fused_qkv", 4, M, K, sum(widths), 128, 0, parts[0].a_bf16,
+                       np.concatenate([p.scales_f16 for p in parts], axis=1),
+                       qweight=np.concatenate([p.qweight for p in parts], axis=1),
+                       qzeros=np.concatenate([p.qzeros for p in parts], axis=1))
+    fused = torch.from_numpy(tf.tf_pack_concat(blobs)).cuda()
+    y = gu.run(whole, kind, blob_dev=fused)
+    gu.check_against_oracle(whole, y)
+    # and column block i of the fused result obeys the acceptance rule of part i on its own
+    n0 = 0
+    for p in parts:
+        gu.check_against_oracle(p, y[:, n0:n0 + p.N].copy())
+        n0 += p.N
