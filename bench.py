@@ -470,6 +470,51 @@ def run_gpu(args):
             del src
         ceilings["note"] = "torch library kernels, same process, context only"
 
+    # ---- ablation (Section 5.5 analogue): fused kernels against full-precision weights kept in memory, and against
+    # dequantizing into memory before every multiplication ------------------------------------------------------
+    ablation = None
+    if rank == 0 and not args.skip_gemm:
+        def timed(fn, n):
+            fn()
+            stream.synchronize()
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record(stream)
+            for _ in range(n):
+                fn()
+            c1.record(stream)
+            stream.synchronize()
+            return c0.elapsed_time(c1) * 1e3 / n
+        ablation = {"note": "us per call; bf16 = torch.matmul on weights held in bf16; unfused = tf_dequant_bf16 into memory, then torch.matmul"}
+        with torch.cuda.stream(stream):
+            for name, M, K, N, fused in (("gemv_1x4096x14336", 1, 4096, 14336, tf.tf_gemv_w4a16),
+                                         ("gemm_2048x4096x14336", 2048, 4096, 14336, tf.tf_gemm_w4a16)):
+                pa = wl.make_w4(M, K, N, seed=7)
+                blobs = [torch.from_numpy(tf.tf_pack_awq(pa.qweight, pa.scales_f16, pa.qzeros, K, N)).to(dev) for _ in range(1)]
+                blobs += [blobs[0].clone() for _ in range(5)]                       # 6 x 29 MB: beyond L2 in rotation
+                a = torch.from_numpy(pa.a_bf16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+                y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                op = tf.TF_OP_GEMV_W4A16 if M <= 16 else tf.TF_OP_GEMM_W4A16
+                aws = torch.zeros(tf.tf_workspace_size(op, M, K, N), dtype=torch.uint8, device=dev)
+                w_full = [torch.empty((K, N), dtype=torch.bfloat16, device=dev) for _ in range(2)]     # 2 x 117 MB
+                tf.tf_dequant_bf16(blobs[0], w_full[0], 4, K, N, stream=stream)
+                w_full[1].copy_(w_full[0])
+                it = {"i": 0}
+                def run_fused():
+                    it["i"] += 1
+                    fused(blobs[it["i"] % 6], a, y, M, K, N, aws, stream=stream)
+                def run_bf16():
+                    it["i"] += 1
+                    torch.matmul(a, w_full[it["i"] & 1], out=y)
+                def run_unfused():
+                    it["i"] += 1
+                    tf.tf_dequant_bf16(blobs[it["i"] % 6], w_full[it["i"] & 1], 4, K, N, stream=stream)
+                    torch.matmul(a, w_full[it["i"] & 1], out=y)
+                n = 30 if M <= 16 else 10
+                ablation[name] = {"fused_w4_us": round(timed(run_fused, n), 2), "bf16_us": round(timed(run_bf16, n), 2),
+                                  "unfused_w4_us": round(timed(run_unfused, n), 2)}
+                assert tf.tf_device_status(aws) == 0
+                del blobs, w_full, a, y, aws
+
     if rank != 0:
         return 0
     cpu_baseline = None
@@ -495,6 +540,7 @@ def run_gpu(args):
         "cpu_baseline": cpu_baseline,
         "per_shape": per_shape,
         "decode_layer": decode_layer,
+        "ablation": ablation,
         "gemm": gemm,
         "ceilings": ceilings,
     }

@@ -154,6 +154,17 @@ tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s_fp16,
 tf_status tf_pack_concat(const void* const* parts, int count, void* out, size_t out_bytes);
 
 /*
+ * Ablation baseline (Sections 4.1 and 5.5): dequantize the whole matrix into global memory, to be
+ * multiplied by a separate full-precision kernel -- the arrangement the fused kernels replace.
+ *   packed   device blob; bits = 4 or 8 must match it.
+ *   w_bf16   device, bf16 [K][N] row-major; receives w[k][n] = bf16((q - z) * s) for W4, bf16(q * s) for
+ *            W8, rounded to nearest even once ((q - z) * s itself is exact in fp32).
+ * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_ALIGN, TF_ERR_ARCH, TF_ERR_CUDA.  A blob whose header does
+ * not match (bits, K, N) leaves w_bf16 untouched.
+ */
+tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int N, void* cuda_stream);
+
+/*
  * Decode-phase fused GEMV (Sections 4.3 "GEMV microkernel" and 4.4): 1 <= M <= 16 tokens.
  *   packed   device, blob from tf_pack_awq (w4a16) / tf_pack_w8 (w8a16) for this K, N.
  *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.

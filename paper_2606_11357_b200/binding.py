@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIG
 
 EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
-           "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static")
+           "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
+           "tf_dequant_bf16")
 
 
 class TileFuseError(RuntimeError):
@@ -54,6 +55,7 @@ def lib() -> ctypes.CDLL:
         L.tf_gemv_w4a16_static.restype = c_int
         L.tf_gemv_w4a16_static.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_workspace_size.restype, L.tf_workspace_size.argtypes = c_size, [c_int] * 4
+        L.tf_dequant_bf16.restype, L.tf_dequant_bf16.argtypes = c_int, [vp, vp, c_int, c_int, c_int, vp]
         L.tf_device_status.restype, L.tf_device_status.argtypes = c_int, [vp, vp]
         L.tf_status_string.restype, L.tf_status_string.argtypes = ctypes.c_char_p, [c_int]
         L.tf_version.restype, L.tf_version.argtypes = c_int, []
@@ -139,6 +141,11 @@ def tf_unpack_w4(packed, q, z, s_f16, K: int, N: int, group_size: int = 128, str
     """packed: uint8 CUDA tensor; q uint8 [K,N], z uint8 [K/g,N], s_f16 float16 [K/g,N] (any may be None)."""
     _check("tf_unpack_w4", lib().tf_unpack_w4(_dev(packed), _dev(q), _dev(z), _dev(s_f16), K, N, group_size,
                                               _stream(stream)))
+
+
+def tf_dequant_bf16(packed, w_bf16, bits: int, K: int, N: int, stream=None) -> None:
+    """packed: uint8 CUDA tensor; w_bf16: bfloat16 CUDA tensor [K, N] that receives the dequantized matrix."""
+    _check("tf_dequant_bf16", lib().tf_dequant_bf16(_dev(packed), _dev(w_bf16), bits, K, N, _stream(stream)))
 
 
 def tf_unpack_w8(packed, q, s_f16, K: int, N: int, group_size: int = 128, stream=None) -> None:

@@ -133,6 +133,21 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_unpack_w8(const v
     return unpack_common(8, packed, q, nullptr, s, K, N, group_size, stream);
 }
 
+extern "C" __attribute__((visibility("default"))) tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int N,
+                                                                           void* stream) {
+    if (!packed || !w_bf16) return TF_ERR_NULL;
+    if (tf_packed_size(bits, K, N, tf::kTileK) == 0) return TF_ERR_SHAPE;
+    if (!aligned16(packed) || !aligned16(w_bf16)) return TF_ERR_ALIGN;
+    DeviceInfo dev;
+    tf_status st = device_info(&dev);
+    if (st != TF_OK) return st;
+    if (tf::launch_dequant(bits, packed, w_bf16, K, N, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return TF_ERR_CUDA;
+    }
+    return TF_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) tf_status tf_device_status(const void* workspace, void* stream) {
     if (!workspace) return TF_ERR_NULL;
     uint32_t word[4] = {0, 0, 0, 0};

@@ -54,6 +54,9 @@ cudaError_t launch_unpack_w4(const void* blob, uint8_t* q, uint8_t* z, uint16_t*
 cudaError_t launch_unpack_w8(const void* blob, int8_t* q, uint16_t* s, int K, int N, int group_size,
                              cudaStream_t stream);
 
+// Ablation baseline: the dequantized matrix written to global memory as bf16 [K][N].
+cudaError_t launch_dequant(int bits, const void* blob, void* w_bf16, int K, int N, cudaStream_t stream);
+
 // Prefill GEMM (tcgen05).  `workspace` starts with the DeviceStatus word.
 size_t gemm_workspace_bytes(int M, int K, int N);
 cudaError_t launch_gemm(int bits, const void* blob, const void* a, void* y, int M, int K, int N,

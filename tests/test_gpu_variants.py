@@ -118,3 +118,22 @@ def test_fused_qkv_blob_from_pack_concat(kind, M):
     for p in parts:
         gu.check_against_oracle(p, y[:, n0:n0 + p.N].copy())
         n0 += p.N
+
+
+@pytest.mark.parametrize("bits,K,N,g", [(4, 512, 200, 128), (4, 1024, 328, 256), (8, 384, 136, 128), (8, 512, 64, 512)])
+def test_dequant_to_memory_is_bit_exact(bits, K, N, g):
+    """The ablation baseline writes w = bf16((q - z) * s) to memory: (q - z) * s is exact in fp32 and in the oracle's
+    fp64, so one round-to-nearest-even of the oracle's value must give the same bits."""
+    p = wl.make_w4(1, K, N, seed=950 + K, group_size=g) if bits == 4 else wl.make_w8(1, K, N, seed=950 + K, group_size=g)
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    guard = 256
+    buf = torch.full((guard + K * N + guard,), gu.CANARY, dtype=torch.int16, device="cuda")
+    w = buf[guard:guard + K * N].view(torch.bfloat16).view(K, N)
+    tf.tf_dequant_bf16(blob, w, bits, K, N)
+    torch.cuda.synchronize()
+    raw = buf.cpu().numpy().view(np.uint16)
+    assert np.all(raw[:guard] == gu.CANARY) and np.all(raw[guard + K * N:] == gu.CANARY), "write outside w"
+    ref = (orc.dequant_w4(p.qweight, p.scales_f16, p.qzeros, g) if bits == 4 else orc.dequant_w8(p.w_i8, p.scales_f16, g))
+    ref32 = ref.astype(np.float32)
+    assert np.array_equal(ref32.astype(np.float64), ref)             # exact in fp32, as claimed
+    assert np.array_equal(raw[guard:guard + K * N].reshape(K, N), wl.f32_to_bf16_bits(ref32))
