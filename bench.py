@@ -548,6 +548,40 @@ def run_gpu(args):
     return 0
 
 
+def run_gemm_sweep(args):
+    """Shape stability of the prefill GEMM (the paper's kernel evaluation, Section 5.1: M swept in steps of 256 over
+    two shapes with K and N swapped).  Prints one JSON object with TFLOP/s per (shape, M)."""
+    import torch
+    from paper_2606_11357_b200 import binding as tf
+    from paper_2606_11357_b200 import workloads as wl
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    rows = []
+    for (K, N) in ((4096, 14336), (14336, 4096)):
+        p = wl.make_w4(1, K, N, seed=11)
+        blob = torch.from_numpy(tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, K, N)).to(dev)
+        for M in range(256, 4097, 256):
+            a = torch.randn((M, K), device=dev).to(torch.bfloat16)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, M, K, N), dtype=torch.uint8, device=dev)
+            for _ in range(3):
+                tf.tf_gemm_w4a16(blob, a, y, M, K, N, ws)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = 10
+            e0.record()
+            for _ in range(n):
+                tf.tf_gemm_w4a16(blob, a, y, M, K, N, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            assert tf.tf_device_status(ws) == 0
+            us = e0.elapsed_time(e1) * 1e3 / n
+            rows.append({"K": K, "N": N, "M": M, "us": round(us, 1), "tflops": round(2.0 * M * K * N / us / 1e6, 1)})
+            del a, y, ws
+    print(json.dumps({"gemm_sweep_w4a16": rows}), flush=True)
+    return 0
+
+
 def run_profile_case(args):
     """A handful of launches of one kernel on one seeded case, for `ncu` captures (prints no bench line)."""
     import torch
@@ -592,7 +626,10 @@ def main(argv=None):
     ap.add_argument("--profile-case", choices=["gemv_w4", "gemv_w4big", "gemv_w8", "gemm_w4", "gemm_w8"], default=None,
                     help="run --steps launches of one kernel on one case and exit (for ncu captures)")
     ap.add_argument("--profile-m", type=int, default=0, help="token count for --profile-case")
+    ap.add_argument("--gemm-sweep", action="store_true", help="time the W4A16 GEMM for M = 256..4096 on two K/N-swapped shapes")
     args = ap.parse_args(argv)
+    if args.gemm_sweep:
+        return run_gemm_sweep(args)
     if args.profile_case:
         return run_profile_case(args)
     if args.warmup < 3:
