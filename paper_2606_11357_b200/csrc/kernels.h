@@ -9,8 +9,11 @@ namespace tf {
 // Up to 8 tokens, short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside
 // this one's and fill their rings while it finishes.  Up to 8 tokens, long ranges: the whole SM, 12 consumer
 // warps and a ring deep enough to keep HBM busy while 12 tiles are being consumed.
-// 9..16 tokens: twice the MMA and activation work per tile, 12 consumer warps and the whole SM.
-__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 12; }
+// 9..16 tokens: twice the MMA and activation work per tile and the whole SM, but 8 consumer warps: a stage carries as
+// many bytes of activations as of weights, so the ring holds half the weights, and every tile a warp is working on is
+// a tile that is not in flight (measured on the four layer shapes: 8 warps 8.4 / 6.0 / 14.6 / 16.7 us, 12 warps
+// 9.4 / 6.4 / 15.9 / 17.0 us, 10 warps in between, 6 and 7 slower).
+__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 8; }
 __host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
 constexpr int kGemvFullFromBytes = 384 * 1024; // packed bytes per CTA from which up to 8 tokens use the whole-SM configuration
