@@ -55,6 +55,11 @@ __host__ __device__ constexpr int act_stages(int bits, int bt) {
                ? kMaxActStages
                : (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt);
 }
+// 64-k sub-steps per pipeline stage.  The thread that issues the MMAs pays a fixed price per stage (two barrier waits,
+// two commits, loop arithmetic on a scheduler it shares with dequant warps): with 64-k stages its loop took about 780
+// cycles per 64 k where the four MMAs of a 256-token tile execute in about 520, and it -- not the tensor core -- set
+// the pace.  Two sub-steps per stage halve that overhead.
+__host__ __device__ constexpr int gemm_substeps(int bits, int bt) { return act_stages(bits, bt) >= 4 ? 2 : 1; }
 constexpr int kEpiWarpBytes = 1024;       // per epilogue warp: 16 tokens x 32 columns of bf16, for the transpose
 constexpr int kDrainWarpBytes = 512;      // per dequant warp: 8 tokens x 32 columns, for its share of an accumulator drain
 __host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
@@ -156,7 +161,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kActStage = act_stage_bytes(BT);
-    constexpr int kStages = act_stages(BITS, BT);
+    constexpr int kSub = gemm_substeps(BITS, BT);
+    constexpr int kStages = act_stages(BITS, BT) / kSub;              // pipeline stages of kSub x 64 k
+    constexpr int kUStage = kSub * kActStage;
+    constexpr int kAU = kAStages / kSub;                              // operand stages of kSub x 32 columns
     constexpr int kWpStripBytes = wp_strip_bytes(BITS);
     constexpr int kWpStageBytes = 2 * kWpStripBytes;
     constexpr uint32_t kIdesc = umma_idesc_bf16(kBN, BT);
@@ -164,7 +172,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* act_ring = smem;                                        // kStages x kActStage   (1024-aligned)
-    uint8_t* wp_ring = act_ring + kStages * kActStage;               // kWpStages x packed tiles
+    uint8_t* wp_ring = act_ring + act_stages(BITS, BT) * kActStage;  // kWpStages x packed tiles
     uint8_t* epi_buf = wp_ring + kWpStages * kWpStageBytes;          // 4 x kEpiWarpBytes
     uint8_t* drain_buf = epi_buf + 4 * kEpiWarpBytes;                // 8 x kDrainWarpBytes
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(drain_buf + 8 * kDrainWarpBytes);
@@ -186,8 +194,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             mbar_init(smem_u32(&bars->act_full[s]), 1);
             mbar_init(smem_u32(&bars->act_empty[s]), 1);     // tcgen05.commit
         }
-        for (int s = 0; s < kAStages; ++s) {
-            mbar_init(smem_u32(&bars->a_full[s]), 4);        // the four dequant warps (lane quarters) of one k-half
+        for (int s = 0; s < kAU; ++s) {
+            mbar_init(smem_u32(&bars->a_full[s]), 4 * kSub); // the dequant warps (lane quarters) of the stage's k-halves
             mbar_init(smem_u32(&bars->a_empty[s]), 1);       // tcgen05.commit
         }
         for (int s = 0; s < kWpStages; ++s) {
@@ -220,13 +228,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 int tile, kt0, len, slot;
                 segs.get(i, tile, kt0, len, slot);
                 const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
-                for (int ks = 2 * kt0; ks < 2 * (kt0 + len); ++ks, ++it) {
+                for (int ks = 2 * kt0; ks < 2 * (kt0 + len); ks += kSub, ++it) {
                     const int s = it % kStages;
                     ok = mbar_wait(smem_u32(&bars->act_empty[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x310 + s);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(smem_u32(&bars->act_full[s]), kActStage);
-                    tma_load_2d(smem_u32(act_ring + s * kActStage), &act_map, ks * kBK, m_tile * BT,
-                                smem_u32(&bars->act_full[s]));
+                    mbar_arrive_expect_tx(smem_u32(&bars->act_full[s]), kUStage);
+#pragma unroll
+                    for (int sub = 0; sub < kSub; ++sub)
+                        tma_load_2d(smem_u32(act_ring + s * kUStage + sub * kActStage), &act_map, (ks + sub) * kBK, m_tile * BT,
+                                    smem_u32(&bars->act_full[s]));
                 }
             }
         } else if (warp == 3 && lane == 0) {
@@ -260,16 +270,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 ok = mbar_wait(smem_u32(&bars->acc_empty), (tile_it & 1) ^ 1, abort_flag, 0x400);
                 if (!ok) break;
                 tc_fence_after();
-                for (int ks = 0; ks < 2 * len; ++ks, ++it) {
-                    const int s = it % kStages, sa = it % kAStages;
-                    ok = mbar_wait(smem_u32(&bars->a_full[sa]), (it / kAStages) & 1, abort_flag, 0x410 + sa) &&
+                for (int ks = 0; ks < 2 * len; ks += kSub, ++it) {
+                    const int s = it % kStages, sa = it % kAU;
+                    ok = mbar_wait(smem_u32(&bars->a_full[sa]), (it / kAU) & 1, abort_flag, 0x410 + sa) &&
                          mbar_wait(smem_u32(&bars->act_full[s]), (it / kStages) & 1, abort_flag, 0x420 + s);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t b_desc = umma_desc_k_sw128(smem_u32(act_ring + s * kActStage));
 #pragma unroll
-                    for (int j = 0; j < kBK / 16; ++j)       // 16 k per instruction: 8 TMEM columns / 32 smem bytes
-                        tc_mma_f16_tmem_a(tmem_base, tmem_a + 32 * sa + 8 * j, b_desc + 2 * j, kIdesc, (ks | j) != 0 ? 1u : 0u);
+                    for (int sub = 0; sub < kSub; ++sub) {
+                        const uint64_t b_desc = umma_desc_k_sw128(smem_u32(act_ring + s * kUStage + sub * kActStage));
+#pragma unroll
+                        for (int j = 0; j < kBK / 16; ++j)   // 16 k per instruction: 8 TMEM columns / 32 smem bytes
+                            tc_mma_f16_tmem_a(tmem_base, tmem_a + 32 * (kSub * sa + sub) + 8 * j, b_desc + 2 * j, kIdesc,
+                                              (ks | sub | j) != 0 ? 1u : 0u);
+                    }
                     tc_commit(smem_u32(&bars->act_empty[s]));
                     tc_commit(smem_u32(&bars->a_empty[sa]));
                 }
@@ -370,14 +384,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars->wp_empty[ws]));
 
-                    // wait until the MMAs that read this operand stage (kAStages steps ago) are done
-                    const uint32_t it = 2 * wit + half;
-                    const int sa = it % kAStages;
-                    ok = mbar_wait(smem_u32(&bars->a_empty[sa]), ((it / kAStages) & 1) ^ 1, abort_flag, 0x510 + sa);
+                    // wait until the MMAs that read this operand stage (kAU stages ago) are done
+                    const uint32_t kstep = 2 * wit + half;                       // 64-k step of this warp's half
+                    const uint32_t it = kstep / kSub;
+                    const int sa = it % kAU;
+                    ok = mbar_wait(smem_u32(&bars->a_empty[sa]), ((it / kAU) & 1) ^ 1, abort_flag, 0x510 + sa);
                     if (!ok) break;
                     tc_fence_after();
                     if (strip_exists) {
-                        const uint32_t taddr = tmem_a + 32 * sa + (uint32_t(32 * q) << 16);
+                        const uint32_t taddr = tmem_a + 32 * (kSub * sa + kstep % kSub) + (uint32_t(32 * q) << 16);
                         tmem_st_16x256b_x4(taddr, op[0]);
                         tmem_st_16x256b_x4(taddr + (16u << 16), op[1]);
                         tmem_st_wait();
