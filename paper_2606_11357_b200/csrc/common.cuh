@@ -81,14 +81,6 @@ __device__ __forceinline__ void mma_bf16_16816(float d[4], uint32_t a0, uint32_t
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
 // Header fields every kernel compares with its arguments (first 24 bytes of the blob).
 __device__ __forceinline__ bool header_matches(const void* blob, uint32_t bits, uint32_t K, uint32_t N) {
     const uint4 h = __ldg(reinterpret_cast<const uint4*>(blob));            // magic, version, bits, K
