@@ -41,7 +41,8 @@ namespace {
 constexpr int kGemmThreads = 512;
 constexpr int kBN = 128;                  // weight columns per CTA tile (two packed strips)
 constexpr int kBK = 64;                   // k per pipeline step (one 128-byte swizzled activation row)
-constexpr int kAStages = 4;               // weight-operand ring in tensor memory (32 columns per k-step)
+constexpr int kMaxDepth = 3;              // pipeline stages (128 k each): activations in shared memory, weight operand in
+                                          // tensor memory (64 columns per stage)
 constexpr int kTmemAccCols = 256;
 constexpr int kTmemCols = 512;
 constexpr int kMaxActStages = 12;
@@ -55,11 +56,11 @@ __host__ __device__ constexpr int act_stages(int bits, int bt) {
                ? kMaxActStages
                : (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt);
 }
-// 64-k sub-steps per pipeline stage.  The thread that issues the MMAs pays a fixed price per stage (two barrier waits,
-// two commits, loop arithmetic on a scheduler it shares with dequant warps): with 64-k stages its loop took about 780
-// cycles per 64 k where the four MMAs of a 256-token tile execute in about 520, and it -- not the tensor core -- set
-// the pace.  Two sub-steps per stage halve that overhead.
-__host__ __device__ constexpr int gemm_substeps(int bits, int bt) { return act_stages(bits, bt) >= 4 ? 2 : 1; }
+// A pipeline stage is 128 k: two 64-k activation sub-tiles and 64 operand columns, one barrier that fills (activations
+// landed + operand stored) and one that drains (MMAs done).  The thread that issues the MMAs pays a fixed price per
+// stage (barrier waits, commits, loop arithmetic on a scheduler it shares with dequant warps): with 64-k stages and
+// separate barriers for the two operands its loop took about 780 cycles per 64 k where the four MMAs of a 256-token
+// tile execute in about 520, and it -- not the tensor core -- set the pace.
 constexpr int kEpiWarpBytes = 1024;       // per epilogue warp: 16 tokens x 32 columns of bf16, for the transpose
 constexpr int kDrainWarpBytes = 512;      // per dequant warp: 8 tokens x 32 columns, for its share of an accumulator drain
 __host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
@@ -108,10 +109,8 @@ struct Segments {
 };
 
 struct GemmBarriers {
-    uint64_t act_full[kMaxActStages];
-    uint64_t act_empty[kMaxActStages];
-    uint64_t a_full[kAStages];
-    uint64_t a_empty[kAStages];
+    uint64_t stage_full[kMaxDepth];       // activations landed (producer's expect_tx) and operand stored (8 dequant warps)
+    uint64_t stage_done[kMaxDepth];       // tcgen05.commit: the MMAs that read the stage have run
     uint64_t wp_full[kWpStages];
     uint64_t wp_empty[kWpStages];
     uint64_t acc_full;
@@ -161,10 +160,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kActStage = act_stage_bytes(BT);
-    constexpr int kSub = gemm_substeps(BITS, BT);
-    constexpr int kStages = act_stages(BITS, BT) / kSub;              // pipeline stages of kSub x 64 k
+    constexpr int kSub = 2;                                           // 64-k sub-steps per pipeline stage
+    constexpr int kStages = act_stages(BITS, BT) / kSub < kMaxDepth ? act_stages(BITS, BT) / kSub : kMaxDepth;
     constexpr int kUStage = kSub * kActStage;
-    constexpr int kAU = kAStages / kSub;                              // operand stages of kSub x 32 columns
+    static_assert(kStages >= 2, "the pipeline needs two stages");
     constexpr int kWpStripBytes = wp_strip_bytes(BITS);
     constexpr int kWpStageBytes = 2 * kWpStripBytes;
     constexpr uint32_t kIdesc = umma_idesc_bf16(kBN, BT);
@@ -191,12 +190,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&bars->act_full[s]), 1);
-            mbar_init(smem_u32(&bars->act_empty[s]), 1);     // tcgen05.commit
-        }
-        for (int s = 0; s < kAU; ++s) {
-            mbar_init(smem_u32(&bars->a_full[s]), 4 * kSub); // the dequant warps (lane quarters) of the stage's k-halves
-            mbar_init(smem_u32(&bars->a_empty[s]), 1);       // tcgen05.commit
+            mbar_init(smem_u32(&bars->stage_full[s]), 9);    // eight dequant warps + the activation producer (with the bytes)
+            mbar_init(smem_u32(&bars->stage_done[s]), 1);    // tcgen05.commit
         }
         for (int s = 0; s < kWpStages; ++s) {
             mbar_init(smem_u32(&bars->wp_full[s]), 1);
@@ -230,13 +225,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
                 for (int ks = 2 * kt0; ks < 2 * (kt0 + len); ks += kSub, ++it) {
                     const int s = it % kStages;
-                    ok = mbar_wait(smem_u32(&bars->act_empty[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x310 + s);
+                    ok = mbar_wait(smem_u32(&bars->stage_done[s]), ((it / kStages) & 1) ^ 1, abort_flag, 0x310 + s);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(smem_u32(&bars->act_full[s]), kUStage);
+                    mbar_arrive_expect_tx(smem_u32(&bars->stage_full[s]), kUStage);
 #pragma unroll
                     for (int sub = 0; sub < kSub; ++sub)
                         tma_load_2d(smem_u32(act_ring + s * kUStage + sub * kActStage), &act_map, (ks + sub) * kBK, m_tile * BT,
-                                    smem_u32(&bars->act_full[s]));
+                                    smem_u32(&bars->stage_full[s]));
                 }
             }
         } else if (warp == 3 && lane == 0) {
@@ -271,9 +266,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 if (!ok) break;
                 tc_fence_after();
                 for (int ks = 0; ks < 2 * len; ks += kSub, ++it) {
-                    const int s = it % kStages, sa = it % kAU;
-                    ok = mbar_wait(smem_u32(&bars->a_full[sa]), (it / kAU) & 1, abort_flag, 0x410 + sa) &&
-                         mbar_wait(smem_u32(&bars->act_full[s]), (it / kStages) & 1, abort_flag, 0x420 + s);
+                    const int s = it % kStages;
+                    ok = mbar_wait(smem_u32(&bars->stage_full[s]), (it / kStages) & 1, abort_flag, 0x410 + s);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
@@ -281,11 +275,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                         const uint64_t b_desc = umma_desc_k_sw128(smem_u32(act_ring + s * kUStage + sub * kActStage));
 #pragma unroll
                         for (int j = 0; j < kBK / 16; ++j)   // 16 k per instruction: 8 TMEM columns / 32 smem bytes
-                            tc_mma_f16_tmem_a(tmem_base, tmem_a + 32 * (kSub * sa + sub) + 8 * j, b_desc + 2 * j, kIdesc,
+                            tc_mma_f16_tmem_a(tmem_base, tmem_a + 32 * (kSub * s + sub) + 8 * j, b_desc + 2 * j, kIdesc,
                                               (ks | sub | j) != 0 ? 1u : 0u);
                     }
-                    tc_commit(smem_u32(&bars->act_empty[s]));
-                    tc_commit(smem_u32(&bars->a_empty[sa]));
+                    tc_commit(smem_u32(&bars->stage_done[s]));
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&bars->acc_full));
@@ -302,7 +295,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
             bool ok = true;
             // Drain duty: every segment's accumulator is released by twelve arrivals, the four epilogue warps and
             // these eight.  For a whole tile a dequant warp first drains its third of its lane quarter.  The duty
-            // for segment s is done just before this warp's third job after the end of s: the first job whose
+            // for segment s is done just before this warp's job number kStages after the end of s: the first job whose
             // operand stage can only be freed by an MMA of segment s + 1, which in turn waits for that release.
             int duty = 0;
             __nv_bfloat16* tbuf8 = reinterpret_cast<__nv_bfloat16*>(drain_buf + (warp - 4) * kDrainWarpBytes);
@@ -326,7 +319,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                 const int n_tile = tile / m_tiles;
                 const bool strip_exists = 2 * n_tile + strip_sel < strips;
                 for (int T = kt0; T < kt0 + len; ++T, ++wit) {
-                    while (ok && (duty < i - 1 || (duty < i && T - kt0 >= 2))) ok = do_duty(duty++);
+                    while (ok && (duty < i - 1 || (duty < i && T - kt0 >= kStages))) ok = do_duty(duty++);
                     if (!ok) break;
                     const int ws = wit % kWpStages;
                     ok = mbar_wait(smem_u32(&bars->wp_full[ws]), (wit / kWpStages) & 1, abort_flag, 0x500 + ws);
@@ -384,22 +377,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars->wp_empty[ws]));
 
-                    // wait until the MMAs that read this operand stage (kAU stages ago) are done
-                    const uint32_t kstep = 2 * wit + half;                       // 64-k step of this warp's half
-                    const uint32_t it = kstep / kSub;
-                    const int sa = it % kAU;
-                    ok = mbar_wait(smem_u32(&bars->a_empty[sa]), ((it / kAU) & 1) ^ 1, abort_flag, 0x510 + sa);
+                    // wait until the MMAs that read this operand stage (kStages stages ago) are done
+                    const uint32_t it = wit;                                     // pipeline stage = k-tile
+                    const int sa = it % kStages;
+                    ok = mbar_wait(smem_u32(&bars->stage_done[sa]), ((it / kStages) & 1) ^ 1, abort_flag, 0x510 + sa);
                     if (!ok) break;
                     tc_fence_after();
                     if (strip_exists) {
-                        const uint32_t taddr = tmem_a + 32 * (kSub * sa + kstep % kSub) + (uint32_t(32 * q) << 16);
+                        const uint32_t taddr = tmem_a + 32 * (kSub * sa + half) + (uint32_t(32 * q) << 16);
                         tmem_st_16x256b_x4(taddr, op[0]);
                         tmem_st_16x256b_x4(taddr + (16u << 16), op[1]);
                         tmem_st_wait();
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[sa]));
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->stage_full[sa]));
                 }
             }
             while (ok && duty < segs.count) ok = do_duty(duty++);
