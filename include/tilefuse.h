@@ -180,7 +180,8 @@ tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int
  * tf_gemv_w8a16 with M <= 2 forms the products in integers: per token and 128-deep k-tile the
  * activations are rewritten on the tile's own power-of-two scale (exact for values within 2^14
  * of the tile's largest magnitude, rounded at 2^-22 of it below that), multiplied with the int8
- * codes exactly in 32 bits, and scaled back in fp32.
+ * codes exactly in 32 bits, and scaled back in fp32.  An Inf or NaN activation makes every output
+ * of its token NaN there (the floating-point paths give Inf or NaN, as IEEE arithmetic does).
  * Each persistent CTA streams one contiguous range of packed tiles; a strip of 64 output
  * columns that is cut between CTAs is summed in CTA order by the last CTA to finish it.
  * The blob must be at least tf_packed_size(bits, K, N, 128) bytes for the K, N passed here.

@@ -453,7 +453,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                             word[0] = __byte_perm(ab01, cd01, 0x5410) ^ 0x80808080u;
                             word[1] = __byte_perm(ab01, cd01, 0x7632) ^ 0x80808080u;
                             word[2] = __byte_perm(ab2, cd2, 0x5410) ^ 0x80808080u;
-                            const float se = __uint_as_float((e - 21u) << 23);             // 2^(emax - 148)
+                            // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
+                            const float se = e == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((e - 21u) << 23);
 #pragma unroll
                             for (int j = 0; j < 3; ++j) {
                                 const int c = 3 * m + j;

@@ -8,6 +8,7 @@ from oracle import tilefuse_oracle as orc
 from paper_2606_11357_b200 import binding as tf
 from paper_2606_11357_b200 import workloads as wl
 import gpu_util as gu
+from helpers import bf16_bits_to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -137,3 +138,19 @@ def test_dequant_to_memory_is_bit_exact(bits, K, N, g):
     ref32 = ref.astype(np.float32)
     assert np.array_equal(ref32.astype(np.float64), ref)             # exact in fp32, as claimed
     assert np.array_equal(raw[guard:guard + K * N].reshape(K, N), wl.f32_to_bf16_bits(ref32))
+
+
+@pytest.mark.parametrize("M", [1, 2, 3])
+def test_w8_gemv_non_finite_activation_is_not_hidden(M):
+    """An Inf or NaN activation must not come out as a finite number: every output of that token is non-finite
+    (NaN on the integer path of 1 and 2 tokens, Inf or NaN on the floating-point path), other tokens are untouched."""
+    K, N = 512, 136
+    p = wl.make_w8(M, K, N, seed=990 + M)
+    clean = gu.run(p, "gemv")
+    bits = p.a_bf16.copy()
+    bits[0, 300] = 0x7F80                      # +Inf in token 0
+    y = gu.run(p, "gemv", a_bits=bits)
+    vals = bf16_bits_to_f64(y)
+    assert not np.any(np.isfinite(vals[0]))
+    if M > 1:
+        assert np.array_equal(y[1:], clean[1:])
