@@ -189,8 +189,14 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     __syncthreads();
     // Programmatic dependent launch: the next kernel on the stream may start as SMs free up.  In this kernel
     // only the packed weights (constants) are read before grid_dependency_wait(); activations, y and the
-    // workspace are touched after it.
-    grid_launch_dependents();
+    // workspace are touched after it.  Whole-SM CTAs release their dependents only when their results are out (the
+    // reducer warp does it after its last strip).  Measured: a half-SM GEMV whose CTAs trickle in behind a whole-SM
+    // one, as its CTAs leave one by one, runs about 11 us late together with the kernels behind it, while the early
+    // release is worth about 2 us between two large whole-SM kernels; the library cannot know which kind follows.
+    // Neither keeping the half-SM kernel out of the early start on its own side nor keeping two of its CTAs off one SM
+    // (by asking for more than half of the shared memory) had any effect, so the cause is not simply two CTAs landing
+    // on one SM.
+    if (!FULL) grid_launch_dependents();
 
     if (warp == 0) {
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
@@ -358,6 +364,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 i += seg_len;
                 ++sidx;
             }
+            if (FULL && lane == 0) grid_launch_dependents();      // whole-SM CTA: its results are out (see above)
         }
     } else if (header_ok) {
         // ---------------- consumers ---------------------------------------------------------------------------
