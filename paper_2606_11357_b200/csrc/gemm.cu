@@ -213,6 +213,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     const uint32_t tmem_base = bars->tmem_base;
     const uint32_t tmem_a = tmem_base + kTmemAccCols;        // weight-operand ring
 
+    // Programmatic dependent launch: this kernel may have been started while the previous kernel of the stream was
+    // still running.  Only the packed weights (constants) are read before grid_dependency_wait(); activations, y and
+    // the workspace are touched after it.  The packed-weight producer is the one role that does not wait here.
+    if (!(warp == 3)) grid_dependency_wait();
+
     if (header_ok) {
         if (warp == 0 && lane == 0) {
             // ================= producer A: activation tile, one TMA load per k-step ==========================
@@ -499,6 +504,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     }
 
     // ---------------- deferred fix-up of the CTA's last cut tile, by all 16 warps --------------------------------
+    if (warp == 3) grid_dependency_wait();
     tc_fence_before();
     __syncthreads();
     if (header_ok && bars->deferred_tile != 0 && bars->abort_flag == 0) {
@@ -557,6 +563,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
 
     // ---------------- teardown --------------------------------------------------------------------------------
     __syncthreads();
+    // this CTA's results are out: the next kernel of the stream may start (a whole-SM kernel releases its dependents
+    // late, see the GEMV)
+    if (threadIdx.x == 0) grid_launch_dependents();
     if (threadIdx.x == 0) {
         if (!header_ok) {
             if (blockIdx.x == 0) { status->code = TF_ERR_BLOB; status->detail = 1; }
@@ -625,10 +634,18 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     const long long tile_cost = (long long)((tiles + tile_grid - 1) / tile_grid) * ktiles;
     const int aligned = tile_cost <= split_cost ? 1 : 0;
     if (aligned) grid = tile_grid;
-    gemm_kernel<BITS, BT><<<grid, kGemmThreads, gemm_smem_bytes(BITS, BT), stream>>>(
-        map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K, N, ktiles, n_tiles, m_tiles, aligned,
-        static_cast<uint8_t*>(workspace));
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = gemm_smem_bytes(BITS, BT);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see grid_dependency_wait() in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_kernel<BITS, BT>, map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K,
+                              N, ktiles, n_tiles, m_tiles, aligned, static_cast<uint8_t*>(workspace));
 }
 
 template <int BITS>
