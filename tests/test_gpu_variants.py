@@ -154,3 +154,31 @@ def test_w8_gemv_non_finite_activation_is_not_hidden(M):
     assert not np.any(np.isfinite(vals[0]))
     if M > 1:
         assert np.array_equal(y[1:], clean[1:])
+
+
+@pytest.mark.parametrize("first,second,M", [("gemv", "gemv", 16), ("gemv", "gemm", 16), ("gemm", "gemm", 96), ("gemm", "gemv", 8)])
+def test_dependent_calls_without_host_sync(first, second, M):
+    """The second call multiplies what the first one writes, on the same stream and workspace, with no host
+    synchronisation in between.  Both kernels are launched so that they may start before their predecessor has
+    finished; they must not read its output early (checked against the oracle applied to the first call's bits)."""
+    K1, N1, N2 = 1024, 1024, 520
+    p1 = wl.make_w4(M, K1, N1, seed=1001, scale_range=(0.002, 0.004))
+    p2 = wl.make_w4(M, N1, N2, seed=1002)
+    b1 = torch.from_numpy(gu.pack(p1)).cuda()
+    b2 = torch.from_numpy(gu.pack(p2)).cuda()
+    a = gu.to_device_bf16(p1.a_bf16)
+    y1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    y2 = torch.empty((M, N2), dtype=torch.bfloat16, device="cuda")
+    ops = {"gemv": (tf.tf_gemv_w4a16, tf.TF_OP_GEMV_W4A16), "gemm": (tf.tf_gemm_w4a16, tf.TF_OP_GEMM_W4A16)}
+    need = max(tf.tf_workspace_size(ops[first][1], M, K1, N1), tf.tf_workspace_size(ops[second][1], M, N1, N2))
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    for _ in range(3):                                   # repeated: an early read would show up intermittently
+        y1.fill_(float("nan"))
+        y2.fill_(float("nan"))
+        ops[first][0](b1, a, y1, M, K1, N1, ws)
+        ops[second][0](b2, y1, y2, M, N1, N2, ws)
+        assert tf.tf_device_status(ws) == 0
+        torch.cuda.synchronize()
+        gu.check_against_oracle(p1, gu.bits_of(y1))
+        p2.a_bf16 = gu.bits_of(y1)
+        gu.check_against_oracle(p2, gu.bits_of(y2))
