@@ -11,6 +11,8 @@
  *   - "host" / "device" on a pointer says which memory it must point into.
  *   - The caller owns every buffer.  The library allocates nothing, frees nothing and
  *     keeps no pointer after a call returns.
+ *     (It remembers, per process, which kind of kernel it launched last on a stream; that
+ *     only steers how consecutive kernels overlap.)
  *   - Device calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*;
  *     NULL = the default stream) and never synchronise, except tf_device_status.
  *   - Errors are return codes.  Nothing is printed, nothing aborts, no exception

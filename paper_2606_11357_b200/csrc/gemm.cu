@@ -644,6 +644,7 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    note_whole_sm_launch(stream);
     return cudaLaunchKernelEx(&cfg, gemm_kernel<BITS, BT>, map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K,
                               N, ktiles, n_tiles, m_tiles, aligned, static_cast<uint8_t*>(workspace));
 }

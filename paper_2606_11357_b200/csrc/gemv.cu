@@ -28,6 +28,8 @@
 // contributor has already published, it fetches their partials while the consumers still work, and the
 // end of the kernel is just one more add.  This keeps the paper's rule that partial sums do not travel
 // between workers for everything but the (at most two) cut strips of a CTA.
+#include <atomic>
+
 #include "async.cuh"
 #include "common.cuh"
 #include "kernels.h"
@@ -189,14 +191,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
     __syncthreads();
     // Programmatic dependent launch: the next kernel on the stream may start as SMs free up.  In this kernel
     // only the packed weights (constants) are read before grid_dependency_wait(); activations, y and the
-    // workspace are touched after it.  Whole-SM CTAs release their dependents only when their results are out (the
-    // reducer warp does it after its last strip).  Measured: a half-SM GEMV whose CTAs trickle in behind a whole-SM
-    // one, as its CTAs leave one by one, runs about 11 us late together with the kernels behind it, while the early
-    // release is worth about 2 us between two large whole-SM kernels; the library cannot know which kind follows.
-    // Neither keeping the half-SM kernel out of the early start on its own side nor keeping two of its CTAs off one SM
-    // (by asking for more than half of the shared memory) had any effect, so the cause is not simply two CTAs landing
-    // on one SM.
-    if (!FULL) grid_launch_dependents();
+    // workspace are touched after it.  (What keeps two half-SM CTAs of one GEMV off the same SM when they come in
+    // behind a whole-SM kernel is decided at launch: see launch_one.)
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
@@ -364,7 +361,6 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 i += seg_len;
                 ++sidx;
             }
-            if (FULL && lane == 0) grid_launch_dependents();      // whole-SM CTA: its results are out (see above)
         }
     } else if (header_ok) {
         // ---------------- consumers ---------------------------------------------------------------------------
@@ -816,6 +812,35 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     return p;
 }
 
+// What this library launched last on a stream: whole-SM kernel or half-SM GEMV.  A scheduling hint only (see
+// launch_one): a stale, missing or raced entry costs overlap between kernels, never correctness.
+namespace {
+constexpr int kLaunchNotes = 8;
+std::atomic<uintptr_t> g_note_stream[kLaunchNotes];
+std::atomic<int> g_note_whole_sm[kLaunchNotes];
+std::atomic<unsigned> g_note_next{0};
+
+bool last_launch_was_half_sm(cudaStream_t stream) {
+    const uintptr_t key = reinterpret_cast<uintptr_t>(stream) + 1;          // 0 = empty slot
+    for (int i = 0; i < kLaunchNotes; ++i)
+        if (g_note_stream[i].load(std::memory_order_relaxed) == key) return g_note_whole_sm[i].load(std::memory_order_relaxed) == 0;
+    return false;
+}
+void note_launch(cudaStream_t stream, bool whole_sm) {
+    const uintptr_t key = reinterpret_cast<uintptr_t>(stream) + 1;
+    for (int i = 0; i < kLaunchNotes; ++i)
+        if (g_note_stream[i].load(std::memory_order_relaxed) == key) {
+            g_note_whole_sm[i].store(whole_sm ? 1 : 0, std::memory_order_relaxed);
+            return;
+        }
+    const int slot = (int)(g_note_next.fetch_add(1, std::memory_order_relaxed) % kLaunchNotes);
+    g_note_whole_sm[slot].store(whole_sm ? 1 : 0, std::memory_order_relaxed);
+    g_note_stream[slot].store(key, std::memory_order_relaxed);
+}
+}  // namespace
+
+void note_whole_sm_launch(cudaStream_t stream) { note_launch(stream, true); }
+
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
@@ -836,7 +861,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     if (unseen) configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             gemv_smem_budget(MT, FULL));
+                                             FULL ? gemv_smem_budget(MT, FULL) : kGemvSoloSmemBytes);
         if (e != cudaSuccess) return e;
         // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
         // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
@@ -851,6 +876,15 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     cfg.blockDim = dim3(p.threads, 1, 1);
     cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = stream;
+    // A whole-SM kernel lets its dependents start as its CTAs leave, one by one.  Every SM freed that way is empty and
+    // takes two half-SM CTAs of the next GEMV while other SMs get none: that kernel then runs on half of the SMs, and
+    // so does every half-SM GEMV behind it, each on the half the one before left free (measured with %smid: 74 SMs
+    // with two CTAs each, 11 us lost per transition, until the next whole-SM kernel).  So a half-SM GEMV that does not
+    // follow another half-SM GEMV of this library on its stream asks for a little more than half of an SM's shared
+    // memory: two of its CTAs no longer fit on one SM, a CTA of the next (plain) half-SM GEMV still fits beside it.
+    if (!FULL && !last_launch_was_half_sm(stream) && cfg.dynamicSmemBytes < (size_t)kGemvSoloSmemBytes)
+        cfg.dynamicSmemBytes = kGemvSoloSmemBytes;
+    note_launch(stream, FULL);
     // Programmatic dependent launch: a CTA uses less than half of an SM (shared memory, registers), so the
     // CTAs of the next GEMV on the stream become resident while this one still runs, fill their rings with
     // weights and then wait for this kernel to finish before they touch activations, y or the workspace.

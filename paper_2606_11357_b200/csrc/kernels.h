@@ -16,6 +16,9 @@ namespace tf {
 __host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 8; }
 __host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
+// Shared memory a half-SM CTA asks for when two of its kind must not share an SM: with 228 KB per SM and 1 KB reserved
+// per CTA, two of these do not fit (2 x 115 KB), one beside a plain half-SM CTA (at most 110 KB) does.
+constexpr int kGemvSoloSmemBytes = 114 * 1024;
 constexpr int kGemvFullFromBytes = 384 * 1024; // packed bytes per CTA from which up to 8 tokens use the whole-SM configuration
 constexpr int kGemvMaxDevices = 64;            // devices the per-device caches cover
 constexpr int kGemvMaxStages = 48;
@@ -51,6 +54,9 @@ struct GemvPlan {
 GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count);
 cudaError_t launch_gemv(int bits, const GemvPlan& plan, const void* blob, const void* a, void* y,
                         int M, int K, int N, void* workspace, cudaStream_t stream);
+
+// Tell the GEMV launcher that a whole-SM kernel of this library (the GEMM) was launched on `stream`.
+void note_whole_sm_launch(cudaStream_t stream);
 
 cudaError_t launch_unpack_w4(const void* blob, uint8_t* q, uint8_t* z, uint16_t* s, int K, int N,
                              int group_size, cudaStream_t stream);
