@@ -182,3 +182,26 @@ def test_dependent_calls_without_host_sync(first, second, M):
         gu.check_against_oracle(p1, gu.bits_of(y1))
         p2.a_bf16 = gu.bits_of(y1)
         gu.check_against_oracle(p2, gu.bits_of(y2))
+
+
+def test_gemv_on_two_streams_with_their_own_workspaces():
+    """Calls on different streams may run concurrently when each stream has its own workspace; what the library
+    remembers about the last launch per stream only steers overlap and must not affect results."""
+    shapes = [(1, 1024, 1024), (16, 1024, 712), (4, 2048, 328), (16, 512, 4096)]
+    probs = [wl.make_w4(M, K, N, seed=1100 + i) for i, (M, K, N) in enumerate(shapes)]
+    blobs = [torch.from_numpy(gu.pack(p)).cuda() for p in probs]
+    acts = [gu.to_device_bf16(p.a_bf16) for p in probs]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    wss = [torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 16, 4096, 4096), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    ys = [[torch.empty((p.M, p.N), dtype=torch.bfloat16, device="cuda") for p in probs] for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(4):
+        for i, p in enumerate(probs):
+            for s in range(2):                            # the same call alternately on the two streams
+                tf.tf_gemv_w4a16(blobs[i], acts[i], ys[s][i], p.M, p.K, p.N, wss[s], stream=streams[s])
+    for s in range(2):
+        assert tf.tf_device_status(wss[s], stream=streams[s]) == 0
+    torch.cuda.synchronize()
+    for i, p in enumerate(probs):
+        gu.check_against_oracle(p, gu.bits_of(ys[0][i]))
+        assert np.array_equal(gu.bits_of(ys[0][i]), gu.bits_of(ys[1][i]))      # same inputs, bit-identical outputs
