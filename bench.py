@@ -251,8 +251,10 @@ def run_gpu(args):
     a_dev_all = [torch.empty(a_elems, dtype=torch.bfloat16, device=dev) for _ in range(2)]
     y_dev_all = [torch.empty(y_elems, dtype=torch.bfloat16, device=dev) for _ in range(2)]
     a_off, y_off = [0, 0], [0, 0]
+    awq_host = {}                                    # the AWQ arrays as given, for the layout arm of the ablation
     for (K, N) in wl.LLAMA3_8B_SHAPES:
         prob = wl.config1(16, K, N)
+        awq_host[(K, N)] = (prob.qweight, prob.scales_f16, prob.qzeros)
         blob_host = tf.tf_pack_awq(prob.qweight, prob.scales_f16, prob.qzeros, K, N)
         a_all = torch.from_numpy(prob.a_bf16.view(np.int16).copy()).view(torch.bfloat16)
         for M in GEMV_MS:
@@ -553,6 +555,46 @@ def run_gpu(args):
                                   "unfused_w4_us": round(timed(run_unfused, n), 2)}
                 assert tf.tf_device_status(aws) == 0
                 del blobs, w_full, a, y, aws
+
+    # ---- layout arm of the ablation: the same fused GEMV on the AWQ arrays as given (no offline pre-tiling) ----
+    if rank == 0 and ablation is not None:
+        layout = {"note": "us per call, graph replay over 6 rotating weight copies (the 2 MB and 9 MB shapes stay in L2 "
+                          "for both arms); pretiled = tf_gemv_w4a16 on the packed blob, raw = tf_gemv_awq_raw on "
+                          "qweight / scales / qzeros"}
+        def replay_us(enqueue, copies):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                enqueue(0)
+                stream.synchronize()
+                with torch.cuda.graph(g, stream=stream):
+                    for c in range(copies):
+                        enqueue(c)
+                g.replay()
+                stream.synchronize()
+                c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                c0.record(stream)
+                for _ in range(5):
+                    g.replay()
+                c1.record(stream)
+                stream.synchronize()
+            return c0.elapsed_time(c1) * 1e3 / (5 * copies)
+        for (K, N) in wl.LLAMA3_8B_SHAPES:
+            qw, sc, qz = awq_host[(K, N)]
+            raw = [(torch.from_numpy(qw.view(np.int32)).to(dev), torch.from_numpy(sc.view(np.int16)).to(dev),
+                    torch.from_numpy(qz.view(np.int32)).to(dev))]
+            raw += [tuple(t.clone() for t in raw[0]) for _ in range(5)]
+            tiled = [next(c[4] for c in calls if (c[2], c[3]) == (K, N))]
+            tiled += [tiled[0].clone() for _ in range(5)]
+            for M in GEMV_MS:
+                a = next(c[5] for c in calls if (c[1], c[2], c[3]) == (M, K, N))
+                y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                rws = torch.empty(tf.tf_gemv_awq_raw_workspace_size(M, K, N, 128), dtype=torch.uint8, device=dev)
+                t_tiled = replay_us(lambda c: tf.tf_gemv_w4a16(tiled[c], a, y, M, K, N, ws, stream=stream), 6)
+                t_raw = replay_us(lambda c: tf.tf_gemv_awq_raw(*raw[c], a, y, M, K, N, 128, rws, stream=stream), 6)
+                layout[f"{M}x{K}x{N}"] = {"pretiled_us": round(t_tiled, 2), "raw_us": round(t_raw, 2)}
+            del raw, tiled
+        assert tf.tf_device_status(ws) == 0
+        ablation["layout"] = layout
 
     if rank != 0:
         return 0

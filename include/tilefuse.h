@@ -241,6 +241,29 @@ tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
 tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_bf16,
                                int M, int K, int N, void* cuda_stream);
 
+/*
+ * Second ablation arm (Section 5.5 separates the gain of fusing from the gain of the offline re-tiling of
+ * Section 4.2): the fused W4A16 GEMV computed straight from the AWQ arrays, without tf_pack_awq.
+ *   qweight     device, uint32 [K][N/8], eight 4-bit codes per word in nibble order 0,2,4,6,1,3,5,7
+ *   scales_fp16 device, fp16 bits [K/group_size][N]
+ *   qzeros      device, uint32 [K/group_size][N/8], same nibble order
+ *   a_bf16      device, bf16 [M][K];  y_bf16  device, bf16 [M][N], fully overwritten
+ *   group_size  32, 64 or 128 (this arm has no tile format to constrain it)
+ *   workspace   device scratch of at least tf_gemv_awq_raw_workspace_size(M, K, N, group_size) bytes
+ *               (fp32 partial sums of the split over K; no initial contents required, no status word).
+ * Arithmetic: (q - z) exact, fp32 multiply-add per group, group sum times the fp16 scale in fp32, fp32
+ * partial sums added in a fixed order, one rounding to bf16.  Two kernel launches on `cuda_stream`.
+ * 1 <= M <= 16; K % group_size == 0; N % 8 == 0; K, N <= TF_MAX_DIM.
+ * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_ALIGN (every device pointer 16-byte aligned),
+ *         TF_ERR_WORKSPACE, TF_ERR_ARCH, TF_ERR_CUDA.
+ */
+tf_status tf_gemv_awq_raw(const uint32_t* qweight, const uint16_t* scales_fp16, const uint32_t* qzeros,
+                          const void* a_bf16, void* y_bf16, int M, int K, int N, int group_size,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* Scratch bytes tf_gemv_awq_raw needs on the current device (0 if the shape is illegal or the device is
+ * not compute capability 10.x). */
+size_t tf_gemv_awq_raw_workspace_size(int M, int K, int N, int group_size);
+
 /* Scratch bytes the given operation needs for this shape (0 if none; 0 also if the shape
  * is illegal -- the compute call then reports TF_ERR_SHAPE). */
 size_t tf_workspace_size(int op, int M, int K, int N);

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIG
 EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
-           "tf_dequant_bf16")
+           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size")
 
 
 class TileFuseError(RuntimeError):
@@ -56,6 +56,9 @@ def lib() -> ctypes.CDLL:
         L.tf_gemv_w4a16_static.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_workspace_size.restype, L.tf_workspace_size.argtypes = c_size, [c_int] * 4
         L.tf_dequant_bf16.restype, L.tf_dequant_bf16.argtypes = c_int, [vp, vp, c_int, c_int, c_int, vp]
+        L.tf_gemv_awq_raw.restype = c_int
+        L.tf_gemv_awq_raw.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, c_int, vp, c_size, vp]
+        L.tf_gemv_awq_raw_workspace_size.restype, L.tf_gemv_awq_raw_workspace_size.argtypes = c_size, [c_int] * 4
         L.tf_device_status.restype, L.tf_device_status.argtypes = c_int, [vp, vp]
         L.tf_status_string.restype, L.tf_status_string.argtypes = ctypes.c_char_p, [c_int]
         L.tf_version.restype, L.tf_version.argtypes = c_int, []
@@ -146,6 +149,19 @@ def tf_unpack_w4(packed, q, z, s_f16, K: int, N: int, group_size: int = 128, str
 def tf_dequant_bf16(packed, w_bf16, bits: int, K: int, N: int, stream=None) -> None:
     """packed: uint8 CUDA tensor; w_bf16: bfloat16 CUDA tensor [K, N] that receives the dequantized matrix."""
     _check("tf_dequant_bf16", lib().tf_dequant_bf16(_dev(packed), _dev(w_bf16), bits, K, N, _stream(stream)))
+
+
+def tf_gemv_awq_raw_workspace_size(M: int, K: int, N: int, group_size: int = 128) -> int:
+    return int(lib().tf_gemv_awq_raw_workspace_size(M, K, N, group_size))
+
+
+def tf_gemv_awq_raw(qweight, scales_f16, qzeros, a, y, M: int, K: int, N: int, group_size: int, workspace,
+                    stream=None) -> None:
+    """The fused GEMV on the AWQ arrays themselves (CUDA tensors: int32 [K, N/8], int16/float16 [K/g, N],
+    int32 [K/g, N/8]); a, y as for tf_gemv_w4a16; workspace: uint8 CUDA tensor."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check("tf_gemv_awq_raw", lib().tf_gemv_awq_raw(_dev(qweight), _dev(scales_f16), _dev(qzeros), _dev(a), _dev(y),
+                                                    M, K, N, group_size, _dev(workspace), ws_bytes, _stream(stream)))
 
 
 def tf_unpack_w8(packed, q, s_f16, K: int, N: int, group_size: int = 128, stream=None) -> None:

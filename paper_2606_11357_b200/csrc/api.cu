@@ -148,6 +148,38 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_dequant_bf16(cons
     return TF_OK;
 }
 
+extern "C" __attribute__((visibility("default"))) size_t tf_gemv_awq_raw_workspace_size(int M, int K, int N, int group_size) {
+    if (M < 1 || M > TF_MAX_M_GEMV || N < 8 || N > TF_MAX_DIM || N % 8 != 0) return 0;
+    if (group_size != 32 && group_size != 64 && group_size != 128) return 0;
+    if (K < group_size || K > TF_MAX_DIM || K % group_size != 0) return 0;
+    DeviceInfo dev;
+    if (device_info(&dev) != TF_OK) return 0;
+    return tf::gemv_raw_workspace_bytes(M, N, dev.sm_count);
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_awq_raw(const uint32_t* qweight, const uint16_t* scales,
+                                                                            const uint32_t* qzeros, const void* a, void* y,
+                                                                            int M, int K, int N, int group_size,
+                                                                            void* workspace, size_t workspace_bytes,
+                                                                            void* stream) {
+    if (!qweight || !scales || !qzeros || !a || !y) return TF_ERR_NULL;
+    if (M < 1 || M > TF_MAX_M_GEMV || N < 8 || N > TF_MAX_DIM || N % 8 != 0) return TF_ERR_SHAPE;
+    if (group_size != 32 && group_size != 64 && group_size != 128) return TF_ERR_SHAPE;
+    if (K < group_size || K > TF_MAX_DIM || K % group_size != 0) return TF_ERR_SHAPE;
+    if (!aligned16(qweight) || !aligned16(scales) || !aligned16(qzeros) || !aligned16(a) || !aligned16(y))
+        return TF_ERR_ALIGN;
+    DeviceInfo dev;
+    tf_status st = device_info(&dev);
+    if (st != TF_OK) return st;
+    if (workspace == nullptr || workspace_bytes < tf::gemv_raw_workspace_bytes(M, N, dev.sm_count)) return TF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return TF_ERR_ALIGN;
+    const tf::RawGemvPlan plan = tf::plan_gemv_raw(K, N, group_size, dev.sm_count);
+    cudaError_t e = tf::launch_gemv_raw(plan, qweight, scales, qzeros, a, y, M, K, N, group_size, workspace,
+                                        static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    return TF_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) tf_status tf_device_status(const void* workspace, void* stream) {
     if (!workspace) return TF_ERR_NULL;
     uint32_t word[4] = {0, 0, 0, 0};

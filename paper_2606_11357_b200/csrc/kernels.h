@@ -66,6 +66,19 @@ cudaError_t launch_unpack_w8(const void* blob, int8_t* q, uint16_t* s, int K, in
 // Ablation baseline: the dequantized matrix written to global memory as bf16 [K][N].
 cudaError_t launch_dequant(int bits, const void* blob, void* w_bf16, int K, int N, cudaStream_t stream);
 
+// Fused W4A16 GEMV on the AWQ arrays as they come (no pre-tiling): the second arm of the layout ablation.
+struct RawGemvPlan {
+    int groups;          // K / group_size
+    int col_blocks;      // blocks of 256 output columns
+    int splits;          // CTAs that share a column block (split-K over whole groups)
+    int groups_per_cta;
+};
+RawGemvPlan plan_gemv_raw(int K, int N, int group_size, int sm_count);
+size_t gemv_raw_workspace_bytes(int M, int N, int sm_count);
+cudaError_t launch_gemv_raw(const RawGemvPlan& plan, const uint32_t* qweight, const uint16_t* scales,
+                            const uint32_t* qzeros, const void* a, void* y, int M, int K, int N, int group_size,
+                            void* workspace, cudaStream_t stream);
+
 // Prefill GEMM (tcgen05).  `workspace` starts with the DeviceStatus word.
 size_t gemm_workspace_bytes(int M, int K, int N);
 cudaError_t launch_gemm(int bits, const void* blob, const void* a, void* y, int M, int K, int N,

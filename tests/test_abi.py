@@ -71,6 +71,14 @@ def test_compute_calls_validate_before_touching_the_gpu():
     assert L.tf_unpack_w4(None, ok, ok, ok, 128, 8, 128, None) == 1
     assert L.tf_unpack_w4(ok, ok, ok, ok, 128, 9, 128, None) == 2
     assert L.tf_device_status(None, None) == 1
+    raw = L.tf_gemv_awq_raw
+    assert raw(None, ok, ok, ok, ok, 1, 128, 8, 128, ok, 1 << 20, None) == 1
+    assert raw(ok, ok, ok, ok, ok, 17, 128, 8, 128, ok, 1 << 20, None) == 2
+    assert raw(ok, ok, ok, ok, ok, 1, 128, 8, 96, ok, 1 << 20, None) == 2       # group size not 32 / 64 / 128
+    assert raw(ok, ok, ok, ok, ok, 1, 160, 8, 64, ok, 1 << 20, None) == 2       # K not a multiple of it
+    assert raw(ok, ok, ok, ok, ok, 1, 128, 12, 128, ok, 1 << 20, None) == 2
+    assert raw(ok, p(0x1004), ok, ok, ok, 1, 128, 8, 128, ok, 1 << 20, None) == 3
+    assert tf.tf_gemv_awq_raw_workspace_size(1, 4096, 4096, 100) == 0
     assert tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 1, 4096, 4096) >= 4096
     assert tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 17, 4096, 4096) == 0
     assert L.tf_gemv_w4a16(ok, ok, ok, 1, 128, 8, None, 0, None) == 5
