@@ -251,8 +251,10 @@ tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_b
  *   group_size  32, 64 or 128 (this arm has no tile format to constrain it)
  *   workspace   device scratch of at least tf_gemv_awq_raw_workspace_size(M, K, N, group_size) bytes
  *               (fp32 partial sums of the split over K; no initial contents required, no status word).
- * Arithmetic: (q - z) exact, fp32 multiply-add per group, group sum times the fp16 scale in fp32, fp32
- * partial sums added in a fixed order, one rounding to bf16.  Two kernel launches on `cuda_stream`.
+ * Arithmetic: (q - z) exact; fp32 multiply-add per group and group sum times the fp16 scale in fp32 (up to 8
+ * tokens), or bf16 x bf16 products of exact operands accumulated in fp32 over 16 rows on the warp MMA and
+ * scaled in fp32 (9 to 16 tokens); fp32 partial sums added in a fixed order, one rounding to bf16.  Two kernel
+ * launches on `cuda_stream`.
  * 1 <= M <= 16; K % group_size == 0; N % 8 == 0; K, N <= TF_MAX_DIM.
  * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_ALIGN (every device pointer 16-byte aligned),
  *         TF_ERR_WORKSPACE, TF_ERR_ARCH, TF_ERR_CUDA.

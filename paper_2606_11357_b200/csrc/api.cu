@@ -173,7 +173,7 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_awq_raw(cons
     if (st != TF_OK) return st;
     if (workspace == nullptr || workspace_bytes < tf::gemv_raw_workspace_bytes(M, N, dev.sm_count)) return TF_ERR_WORKSPACE;
     if (!aligned16(workspace)) return TF_ERR_ALIGN;
-    const tf::RawGemvPlan plan = tf::plan_gemv_raw(K, N, group_size, dev.sm_count);
+    const tf::RawGemvPlan plan = tf::plan_gemv_raw(M, K, N, group_size, dev.sm_count);
     cudaError_t e = tf::launch_gemv_raw(plan, qweight, scales, qzeros, a, y, M, K, N, group_size, workspace,
                                         static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }

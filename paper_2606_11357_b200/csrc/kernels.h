@@ -68,12 +68,13 @@ cudaError_t launch_dequant(int bits, const void* blob, void* w_bf16, int K, int 
 
 // Fused W4A16 GEMV on the AWQ arrays as they come (no pre-tiling): the second arm of the layout ablation.
 struct RawGemvPlan {
-    int groups;          // K / group_size
-    int col_blocks;      // blocks of 256 output columns
-    int splits;          // CTAs that share a column block (split-K over whole groups)
+    bool mma;            // 3..16 tokens: tensor-core kernel (units are 16-row blocks); else the fp32 kernel (units are groups)
+    int groups;          // units along K
+    int col_blocks;      // blocks of 256 (fp32) or 64 (tensor-core) output columns
+    int splits;          // CTAs that share a column block (split-K over whole units)
     int groups_per_cta;
 };
-RawGemvPlan plan_gemv_raw(int K, int N, int group_size, int sm_count);
+RawGemvPlan plan_gemv_raw(int M, int K, int N, int group_size, int sm_count);
 size_t gemv_raw_workspace_bytes(int M, int N, int sm_count);
 cudaError_t launch_gemv_raw(const RawGemvPlan& plan, const uint32_t* qweight, const uint16_t* scales,
                             const uint32_t* qzeros, const void* a, void* y, int M, int K, int N, int group_size,

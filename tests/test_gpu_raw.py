@@ -34,7 +34,7 @@ def run_raw(p, a_bits=None):
 
 
 SHAPES = [(1, 128, 8), (1, 256, 64), (2, 256, 72), (3, 384, 200), (4, 512, 256), (5, 640, 264), (8, 1024, 1000),
-          (9, 512, 136), (16, 1152, 320), (1, 8192, 8), (16, 4096, 64), (7, 2048, 2056)]
+          (9, 512, 136), (16, 1152, 320), (1, 8192, 8), (16, 4096, 64), (7, 2048, 2056), (12, 640, 328)]
 
 
 @pytest.mark.parametrize("M,K,N", SHAPES)
