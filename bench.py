@@ -509,6 +509,29 @@ def run_gpu(args):
             stream.synchronize()
             ceilings["read_only_pass_gbs"] = round(src.numel() * 4 / (c0.elapsed_time(c1) * 1e3 / 5) / 1e3, 1)
             del src
+            # a device-to-device copy of as many bytes as each GEMV shape reads, back to back in a graph over rotating
+            # sources: what a dependent chain of trivial kernels of that size takes (it moves twice the bytes)
+            chain = {}
+            for nbytes in sorted({gemv_algorithmic_bytes(4, 1, K, N) for (K, N) in wl.LLAMA3_8B_SHAPES}):
+                copies = max(4, int(300e6 // nbytes) + 1)
+                srcs = [torch.empty(nbytes // 4, dtype=torch.float32, device=dev).zero_() for _ in range(copies)]
+                dst = torch.empty(nbytes // 4, dtype=torch.float32, device=dev)
+                g = torch.cuda.CUDAGraph()
+                dst.copy_(srcs[0])
+                stream.synchronize()
+                with torch.cuda.graph(g, stream=stream):
+                    for t in srcs:
+                        dst.copy_(t)
+                g.replay()
+                stream.synchronize()
+                c0.record(stream)
+                for _ in range(5):
+                    g.replay()
+                c1.record(stream)
+                stream.synchronize()
+                chain[str(nbytes)] = round(c0.elapsed_time(c1) * 1e3 / (5 * copies), 2)
+                del g, srcs, dst
+            ceilings["copy_us_per_call_at_gemv_bytes"] = chain
         ceilings["note"] = "torch library kernels, same process, context only"
 
     # ---- ablation (Section 5.5 analogue): fused kernels against full-precision weights kept in memory, and against
