@@ -129,6 +129,36 @@ def test_config1_decode_sweep(M, K, N):
     gu.check_against_oracle(p, gu.run(p, "gemv"))
 
 
+def test_config1_step_replayed_as_one_graph():
+    """The twelve calls of the decode step the way the benchmark issues them: one stream, one workspace, captured
+    once into a CUDA graph and replayed, every kernel free to start under its predecessor's tail.  Every result is
+    checked against the oracle on the first and last columns and a seeded sample in between."""
+    probs = [wl.config1(M, K, N) for M in (1, 4, 16) for (K, N) in wl.LLAMA3_8B_SHAPES]
+    packed = [torch.from_numpy(gu.pack(p)).cuda() for p in probs]
+    acts = [gu.to_device_bf16(p.a_bf16) for p in probs]
+    ys = [torch.full((p.M, p.N), float("nan"), dtype=torch.bfloat16, device="cuda") for p in probs]
+    ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 16, 4096, 4096), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        for p, b, a, y in zip(probs, packed, acts, ys):            # first use outside the capture
+            tf.tf_gemv_w4a16(b, a, y, p.M, p.K, p.N, ws, stream=stream)
+        stream.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            for p, b, a, y in zip(probs, packed, acts, ys):
+                tf.tf_gemv_w4a16(b, a, y, p.M, p.K, p.N, ws, stream=stream)
+        for y in ys:
+            y.fill_(float("nan"))
+        for _ in range(3):
+            graph.replay()
+        stream.synchronize()
+    assert tf.tf_device_status(ws) == 0
+    rng = np.random.default_rng(17)
+    for p, y in zip(probs, ys):
+        cols = np.unique(np.concatenate([np.arange(0, 8), np.arange(p.N - 8, p.N), rng.integers(0, p.N, size=48)]))
+        gu.check_against_oracle(p, gu.bits_of(y), columns=cols)
+
+
 def test_config3_w8_gemv():
     p = wl.config3_gemv()
     gu.check_against_oracle(p, gu.run(p, "gemv"))
