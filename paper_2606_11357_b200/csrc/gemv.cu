@@ -123,12 +123,16 @@ __device__ __forceinline__ void store_strip(__nv_bfloat16* y, const float4 (&tot
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
-                   __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
+                   const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
                    int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes,
                    uint8_t* __restrict__ workspace) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
+    // 9..16 tokens: a stage would carry as many bytes of activations as of weights and the ring would hold half the
+    // weights.  There the consumer warps read their activation fragments straight from global memory (L2) instead,
+    // issued before they wait for the tile's weights, and the ring is all weights.
+    constexpr bool kActFromGlobal = !I8;
     constexpr int kActOffset = kGemvActOffset;            // activations sit behind the weights of a stage
     constexpr int kTok = 8 * MT;
     constexpr int kVecPerKb = BITS == 4 ? 1 : 2;
@@ -202,7 +206,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
         // dozen instructions per chunk: this warp shares its scheduler with consumer warps that never idle.
         if (lane == 0 && header_ok) {
             prefetch_tensormap(&act_map);
-            const uint32_t act_bytes = (uint32_t)M * 128u * 2u * kR;
+            const uint32_t act_bytes = kActFromGlobal ? 0u : (uint32_t)M * 128u * 2u * kR;
             ChunkWalk walk(t0, ntiles, ktiles, blob + kHeaderBytes, kTileBytes);
             // first ring fill, weights only: they are constants, so they may be fetched before the dependency wait
             int cg = 0;
@@ -222,7 +226,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     int tiles_here, T;
                     const uint8_t* src;
                     again.next(kR, tiles_here, T, src);
-                    tma_load_3d(smem_u32(ring + (size_t)c * stage_bytes) + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * c);
+                    if (!kActFromGlobal)
+                        tma_load_3d(smem_u32(ring + (size_t)c * stage_bytes) + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * c);
                 }
             }
             // everything else in ring order
@@ -237,7 +242,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 stage_tag[s] = (uint32_t)cg;                 // the stage's previous use is fully consumed by now
                 mbar_arrive_expect_tx(full0 + 8 * s, (uint32_t)tiles_here * kTileBytes + act_bytes);
                 bulk_copy_g2s(dst, src, (uint32_t)tiles_here * kTileBytes, full0 + 8 * s);
-                tma_load_3d(dst + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * s);
+                if (!kActFromGlobal) tma_load_3d(dst + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * s);
                 if (++s == nstages) { s = 0; parity ^= 1u; }
             }
         }
@@ -392,6 +397,18 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 cg_cur = cg;
                 while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
                 const int s = s_cur;
+                uint2 ag[kActFromGlobal ? MT : 1][kActFromGlobal ? 8 : 1];     // token g (+8): k = 128 T + 16 kb + 4t .. +3
+                if constexpr (kActFromGlobal) {
+                    const __nv_bfloat16* arow = a_glob + (size_t)(T0 + lj) * kTileK + 4 * t;
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int kb = 0; kb < 8; ++kb) {
+                            ag[mt][kb] = make_uint2(0u, 0u);
+                            if (g + 8 * mt < M)
+                                ag[mt][kb] = __ldg(reinterpret_cast<const uint2*>(arow + (size_t)(g + 8 * mt) * K + 16 * kb));
+                        }
+                }
                 if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
                     const long long t_begin = clock64();
                     while (stage_tag[s] != (uint32_t)cg && !aborted) {
@@ -541,8 +558,12 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        av[mt] = make_uint2(0u, 0u);
-                        if (g + 8 * mt < M) av[mt] = lds_v2(abase[mt][kb >> 2] ^ ((kb & 3) << 5));
+                        if constexpr (kActFromGlobal) {
+                            av[mt] = ag[mt][kb];
+                        } else {
+                            av[mt] = make_uint2(0u, 0u);
+                            if (g + 8 * mt < M) av[mt] = lds_v2(abase[mt][kb >> 2] ^ ((kb & 3) << 5));
+                        }
                     }
                     uint4 wv[kVecPerKb];
 #pragma unroll
@@ -797,7 +818,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
     const int kr = gemv_chunk_tiles(bits);
     // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
-    p.stage_bytes = kGemvActOffset + ((M * 128 * 2 * kr + 1023) / 1024) * 1024;
+    p.stage_bytes = kGemvActOffset + (!(bits == 8 && M <= kGemvI8MaxM) ? 0 : ((M * 128 * 2 * kr + 1023) / 1024) * 1024);   // 9..16 tokens: activations are read from global memory
     // cluster mode: one slot per CTA of the cluster for the rows of real tokens (two token rows = 512 bytes)
     p.xslot_bytes = p.cluster > 1 ? ((M + 1) / 2) * 512 : 0;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4 +
@@ -899,7 +920,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
         cfg.numAttrs = 2;
     }
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8>, map, static_cast<const uint8_t*>(blob),
-                              static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
+                              static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
                               p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace));
 }
 
