@@ -4,14 +4,20 @@
 // contiguous payload carrying its scales and zeros, strip after strip).  That sequence is cut into
 // equal contiguous ranges, one per CTA, so every CTA streams one contiguous byte range of HBM:
 //
-//   producer warp : one lane issues, per ring stage, one bulk (TMA) copy of several consecutive tiles
-//                   and one tiled TMA load of the activations those tiles multiply (M x 128 k per tile,
-//                   128-byte swizzled); completion on mbarriers.  Bytes in flight are bounded by the
-//                   ring, not by registers, and no consumer ever waits on a global load.  One lane with
-//                   a short loop is enough: a lone lane streams 16 KB copies at the full HBM rate, while
-//                   several lanes of one warp only take turns, and every instruction of this warp
-//                   competes for issue slots with consumer warps that never idle.
-//   consumer warps: take tiles round-robin; 128-bit shared loads, codes -> exact small-integer bf16
+//   producer warp : one lane issues, per ring stage, one bulk (TMA) copy of several consecutive tiles;
+//                   completion on mbarriers.  Weight bytes in flight are bounded by the ring, not by
+//                   registers.  One lane with a short loop is enough: a lone lane streams 16 KB copies at
+//                   the full HBM rate, while several lanes of one warp only take turns, and every
+//                   instruction of this warp competes for issue slots with consumer warps that never idle.
+//                   It reads nothing but weights, which are constants, so it does not wait for earlier
+//                   kernels of the stream.
+//   consumer warps: take tiles round-robin.  A warp first asks for the tile's activations -- its own MMA
+//                   fragment, 8 bytes per lane and 16-k block (integer path: its 4 k of the tile's 128 per
+//                   token), straight from global memory (they sit in
+//                   L2) -- and only then waits for the tile's weights, so the two latencies overlap and the
+//                   ring holds nothing but weights (staging activations through the ring put a TMA load
+//                   behind the dependency wait of every call, about 1 us, and took ring space from the
+//                   weights: half of it for 9..16 tokens).  128-bit shared loads, codes -> exact small-integer bf16
 //                   (q - z), contraction with the activations on the warp-level tensor-core MMA
 //                   (weights = the 16x16 operand, up to 8 tokens = the 16x8 operand: the per-weight
 //                   cost does not grow with M), fp16 scale applied in fp32 once per group.
@@ -33,21 +39,10 @@
 #include "async.cuh"
 #include "common.cuh"
 #include "kernels.h"
-#include "tensormap.h"
 
 namespace tf {
 
 namespace {
-
-__device__ __forceinline__ void consumer_bar_sync(int nthreads) {
-    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
-}
-
-__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-    return v;
-}
 
 // Integer warp MMA: D(16x8, s32) += A(16x32, s8) . B(32x8, s8).  Thread (g, t): a0 = row g, k 4t..4t+3; a1 = row g+8;
 // a2, a3 = the same rows, k + 16; b0 = column g, k 4t..4t+3; b1 = k + 16; d = rows g, g+8 x columns 2t, 2t+1.
@@ -122,18 +117,12 @@ __device__ __forceinline__ void store_strip(__nv_bfloat16* y, const float4 (&tot
 
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
-gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
-                   const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
+gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
                    int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes,
                    uint8_t* __restrict__ workspace) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
-    // 9..16 tokens: a stage would carry as many bytes of activations as of weights and the ring would hold half the
-    // weights.  There the consumer warps read their activation fragments straight from global memory (L2) instead,
-    // issued before they wait for the tile's weights, and the ring is all weights.
-    constexpr bool kActFromGlobal = !I8;
-    constexpr int kActOffset = kGemvActOffset;            // activations sit behind the weights of a stage
     constexpr int kTok = 8 * MT;
     constexpr int kVecPerKb = BITS == 4 ? 1 : 2;
     constexpr int kRedWarp = kTok * kTileN;               // floats one consumer warp drops per strip segment
@@ -201,12 +190,11 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
 
     if (warp == 0) {
         // ---------------- producer: stream this CTA's contiguous tile range through the ring --------------
-        // One lane issues, per chunk, one bulk copy of up to kR contiguous tiles of one strip plus one tensor copy
-        // of the activations of those k-tiles.  Chunks never straddle a strip boundary.  The loop is kept to a few
-        // dozen instructions per chunk: this warp shares its scheduler with consumer warps that never idle.
+        // One lane issues, per chunk, one bulk copy of up to kR contiguous tiles of one strip.  Chunks never straddle
+        // a strip boundary.  The loop is kept to a few dozen instructions per chunk: this warp shares its scheduler
+        // with consumer warps that never idle.  It reads nothing but the packed weights, which are constants, so it
+        // does not wait for the kernels before this one: the first ring fill is on its way while they finish.
         if (lane == 0 && header_ok) {
-            prefetch_tensormap(&act_map);
-            const uint32_t act_bytes = kActFromGlobal ? 0u : (uint32_t)M * 128u * 2u * kR;
             ChunkWalk walk(t0, ntiles, ktiles, blob + kHeaderBytes, kTileBytes);
             // first ring fill, weights only: they are constants, so they may be fetched before the dependency wait
             int cg = 0;
@@ -215,20 +203,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 const uint8_t* src;
                 walk.next(kR, tiles_here, T, src);
                 stage_tag[cg] = (uint32_t)cg;
-                mbar_arrive_expect_tx(full0 + 8 * cg, (uint32_t)tiles_here * kTileBytes + act_bytes);
+                mbar_arrive_expect_tx(full0 + 8 * cg, (uint32_t)tiles_here * kTileBytes);
                 bulk_copy_g2s(smem_u32(ring + (size_t)cg * stage_bytes), src, (uint32_t)tiles_here * kTileBytes, full0 + 8 * cg);
-            }
-            const int nfill = cg;
-            grid_dependency_wait();
-            {   // the activations of the first fill
-                ChunkWalk again(t0, ntiles, ktiles, blob + kHeaderBytes, kTileBytes);
-                for (int c = 0; c < nfill; ++c) {
-                    int tiles_here, T;
-                    const uint8_t* src;
-                    again.next(kR, tiles_here, T, src);
-                    if (!kActFromGlobal)
-                        tma_load_3d(smem_u32(ring + (size_t)c * stage_bytes) + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * c);
-                }
             }
             // everything else in ring order
             int s = 0;
@@ -240,9 +216,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 walk.next(kR, tiles_here, T, src);
                 const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
                 stage_tag[s] = (uint32_t)cg;                 // the stage's previous use is fully consumed by now
-                mbar_arrive_expect_tx(full0 + 8 * s, (uint32_t)tiles_here * kTileBytes + act_bytes);
+                mbar_arrive_expect_tx(full0 + 8 * s, (uint32_t)tiles_here * kTileBytes);
                 bulk_copy_g2s(dst, src, (uint32_t)tiles_here * kTileBytes, full0 + 8 * s);
-                if (!kActFromGlobal) tma_load_3d(dst + kActOffset, &act_map, 0, 2 * T, 0, full0 + 8 * s);
                 if (++s == nstages) { s = 0; parity ^= 1u; }
             }
         }
@@ -397,8 +372,16 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 cg_cur = cg;
                 while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
                 const int s = s_cur;
-                uint2 ag[kActFromGlobal ? MT : 1][kActFromGlobal ? 8 : 1];     // token g (+8): k = 128 T + 16 kb + 4t .. +3
-                if constexpr (kActFromGlobal) {
+                uint2 araw[2];                                  // integer path: token m, k = 128 T + 4 lane .. +3
+                if constexpr (I8) {
+#pragma unroll
+                    for (int m = 0; m < 2; ++m) {
+                        araw[m] = make_uint2(0u, 0u);
+                        if (m < M) araw[m] = __ldg(reinterpret_cast<const uint2*>(a_glob + (size_t)m * K + (size_t)(T0 + lj) * kTileK + 4 * lane));
+                    }
+                }
+                uint2 ag[!I8 ? MT : 1][!I8 ? 8 : 1];            // token g (+8): k = 128 T + 16 kb + 4t .. +3
+                if constexpr (!I8) {
                     const __nv_bfloat16* arow = a_glob + (size_t)(T0 + lj) * kTileK + 4 * t;
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt)
@@ -420,18 +403,6 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                 if (!mbar_wait(full0 + 8 * s, use_cur & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
                 const uint8_t* stage = ring + (size_t)s * stage_bytes;
                 const uint8_t* tile = stage + (size_t)slot * kTileBytes;
-                // activations of this k-tile in the stage: rows of 64 k (128 B), row index = m * 2kR + kc with
-                // kc = 2 * slot + (kb >> 2), 16-byte chunks XOR-swizzled with (row & 7)
-                // shared address of 16-byte chunk 0 of this lane's two rows (k 0..63, 64..127) per token tile, with the
-                // swizzle key folded in: chunk c of the row is at (address ^ (c << 5))
-                uint32_t abase[MT][2];
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int row = (g + 8 * mt) * (2 * kR) + 2 * slot + h;
-                        abase[mt][h] = smem_u32(stage + kActOffset) + row * 128 + ((((row & 7) ^ (t >> 1))) << 4) + (t & 1) * 8;
-                    }
 
                 const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
                 if constexpr (I8) {
@@ -452,9 +423,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     for (int m = 0; m < 2; ++m) {
                         if (m < M) {
                             // lane L holds k = 4L .. 4L+3 of the tile
-                            const int row = m * (2 * kR) + 2 * slot + (lane >> 4);
-                            const uint2 raw = lds_v2(smem_u32(stage + kActOffset) + row * 128 +
-                                                     (((((lane & 15) >> 1) ^ (row & 7))) << 4) + (lane & 1) * 8);
+                            const uint2 raw = araw[m];
                             const uint32_t x0 = raw.x, x1 = raw.y;
                             uint32_t e = max(max((x0 << 17) >> 24, (x0 << 1) >> 24), max((x1 << 17) >> 24, (x1 << 1) >> 24));
                             e = __reduce_max_sync(0xFFFFFFFFu, e);
@@ -558,12 +527,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* _
                     uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        if constexpr (kActFromGlobal) {
-                            av[mt] = ag[mt][kb];
-                        } else {
-                            av[mt] = make_uint2(0u, 0u);
-                            if (g + 8 * mt < M) av[mt] = lds_v2(abase[mt][kb >> 2] ^ ((kb & 3) << 5));
-                        }
+                        av[mt] = ag[mt][kb];
                     }
                     uint4 wv[kVecPerKb];
 #pragma unroll
@@ -817,8 +781,8 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     if (tiles_per_cta < p.consumers) p.consumers = tiles_per_cta < 4 ? 4 : tiles_per_cta;
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
     const int kr = gemv_chunk_tiles(bits);
-    // a stage: kR packed tiles (padded to kGemvActOffset) + the activations of those k-tiles, 1024-aligned
-    p.stage_bytes = kGemvActOffset + (!(bits == 8 && M <= kGemvI8MaxM) ? 0 : ((M * 128 * 2 * kr + 1023) / 1024) * 1024);   // 9..16 tokens: activations are read from global memory
+    // a stage: one bulk copy of kR packed tiles, padded to a multiple of 1 KB
+    p.stage_bytes = kGemvStageBytes;
     // cluster mode: one slot per CTA of the cluster for the rows of real tokens (two token rows = 512 bytes)
     p.xslot_bytes = p.cluster > 1 ? ((M + 1) / 2) * 512 : 0;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4 +
@@ -865,14 +829,6 @@ void note_whole_sm_launch(cudaStream_t stream) { note_launch(stream, true); }
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
-    // activations [M][K] seen as {64 k, K/64, M tokens} (strides increase with the dimension): one box = the
-    // M x (128 k x kR) slab of a ring stage, landing in shared memory as [token][k-chunk of 64][64 k]
-    CUtensorMap map;
-    const cuuint64_t dims[3] = {64, (cuuint64_t)K / 64, (cuuint64_t)M};
-    const cuuint64_t strides[2] = {128, (cuuint64_t)K * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)(2 * gemv_chunk_tiles(BITS)), (cuuint32_t)M};
-    cudaError_t me = encode_bf16_map(&map, a, 3, dims, strides, box);
-    if (me != cudaSuccess) return me;
     // function attributes belong to one device: set them once per device and kernel (twice is harmless)
     static bool configured_on[kGemvMaxDevices] = {};
     int dev = 0;
@@ -919,7 +875,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
         attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
         cfg.numAttrs = 2;
     }
-    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8>, map, static_cast<const uint8_t*>(blob),
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8>, static_cast<const uint8_t*>(blob),
                               static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
                               p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace));
 }

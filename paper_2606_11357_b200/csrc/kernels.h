@@ -9,10 +9,9 @@ namespace tf {
 // Up to 8 tokens, short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside
 // this one's and fill their rings while it finishes.  Up to 8 tokens, long ranges: the whole SM, 12 consumer
 // warps and a ring deep enough to keep HBM busy while 12 tiles are being consumed.
-// 9..16 tokens: twice the MMA and activation work per tile and the whole SM, but 8 consumer warps: a stage carries as
-// many bytes of activations as of weights, so the ring holds half the weights, and every tile a warp is working on is
-// a tile that is not in flight (measured on the four layer shapes: 8 warps 8.4 / 6.0 / 14.6 / 16.7 us, 12 warps
-// 9.4 / 6.4 / 15.9 / 17.0 us, 10 warps in between, 6 and 7 slower).
+// 9..16 tokens: twice the MMA and activation work per tile and the whole SM, but 8 consumer warps: every tile a warp
+// is working on is a tile that is not in flight (measured on the four layer shapes with the ring holding weights only:
+// 8 warps 7.9 / 4.1 / 14.5 / 15.4 us, 10 warps 8.4 / 4.1 / 15.2 / 16.1 us; 12 warps do not fit the register file).
 __host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 8; }
 __host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
@@ -24,10 +23,9 @@ constexpr int kGemvMaxDevices = 64;            // devices the per-device caches 
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
 constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (<= K/128 + 1 = 257)
-// A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way), padded to
-// kGemvActOffset, followed by the activations of the same k-tiles.
+// A ring stage holds one bulk copy of several contiguous tiles (about 16.6 KB either way).
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
-constexpr int kGemvActOffset = 17408;         // 17 x 1024 >= 4 x 4256 and >= 2 x 8320
+constexpr int kGemvStageBytes = 17408;        // 17 x 1024 >= 4 x 4256 and >= 2 x 8320
 constexpr int kGemvMaxM = 16;
 constexpr int kGemvI8MaxM = 2;                // int8 weights, up to this many tokens: the GEMV runs on the integer warp MMA
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
@@ -46,7 +44,7 @@ struct GemvPlan {
     int cluster;       // CTAs per cluster (1 = global mode: cut strips go through the workspace)
     int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster); global mode: CTAs that get tiles
     int xslot_bytes;   // cluster mode: bytes of one partial-sum slot in shared memory
-    int stage_bytes;   // bytes of one ring stage (weights + activations)
+    int stage_bytes;   // bytes of one ring stage
     int smem_bytes;
     int strips, ktiles, total_tiles;
 };
