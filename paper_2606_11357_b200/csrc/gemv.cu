@@ -773,7 +773,8 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     }
     // Long ranges amortise the start of the kernel: take the whole SM (more consumer warps, deeper ring).  Short
     // ones gain more from the next GEMV's CTAs sitting beside this one's with their rings already full.
-    p.full = mt == 2 || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= kGemvFullFromBytes;
+    const bool i8_path = bits == 8 && M <= kGemvI8MaxM;
+    p.full = mt == 2 || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= (i8_path ? kGemvFullFromBytesI8 : kGemvFullFromBytes);
     p.i8 = bits == 8 && M <= kGemvI8MaxM && p.cluster == 1;
     // the integer path leaves the warps waiting for data, not for issue slots: 8 of them keep more tiles in flight
     // (4096x14336, 1 token: 13.7 us with 8 warps, 14.2 us with 12)

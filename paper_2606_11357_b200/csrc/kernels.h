@@ -18,7 +18,14 @@ __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (
 // Shared memory a half-SM CTA asks for when two of its kind must not share an SM: with 228 KB per SM and 1 KB reserved
 // per CTA, two of these do not fit (2 x 115 KB), one beside a plain half-SM CTA (at most 110 KB) does.
 constexpr int kGemvSoloSmemBytes = 114 * 1024;
-constexpr int kGemvFullFromBytes = 384 * 1024; // packed bytes per CTA from which up to 8 tokens use the whole-SM configuration
+// Packed bytes per CTA from which up to 8 tokens use the whole-SM configuration.  Measured with the same call back
+// to back, the whole SM wins from about 400 KB (4096 x 28672: 18.1 against 19.4 us); between calls of other sizes
+// the half-SM form overlaps with its neighbours and wins up to more (a decoder layer whose joined gate + up
+// projection has 412 KB per CTA: 41.2 against 46.8 us per layer).  At 472 KB (4096 x 32768) the whole SM is ahead
+// by 2 us either way.  The integer path has 8 consumer warps in both forms and crosses over later (562 KB per
+// CTA: 16.6 us half, 17.7 whole; 787 KB: 23.1 / 22.7; 899 KB: 30.7 / 26.0).
+constexpr int kGemvFullFromBytes = 440 * 1024;
+constexpr int kGemvFullFromBytesI8 = 704 * 1024;
 constexpr int kGemvMaxDevices = 64;            // devices the per-device caches cover
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
