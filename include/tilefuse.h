@@ -168,7 +168,11 @@ tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int
 
 /*
  * Decode-phase fused GEMV (Sections 4.3 "GEMV microkernel" and 4.4): 1 <= M <= 16 tokens.
- *   packed   device, blob from tf_pack_awq (w4a16) / tf_pack_w8 (w8a16) for this K, N.
+ *   packed   device, blob from tf_pack_awq (w4a16) / tf_pack_w8 (w8a16) for this K, N.  Weights are treated
+ *            as constants: the kernels start fetching them before the stream's earlier kernels have finished
+ *            where those release their dependents early (programmatic dependent launch, as this library's
+ *            own kernels do).  Ordinary stream order covers a blob written by a copy or by a kernel that does
+ *            not do that; activations, results and the workspace are always touched in stream order.
  *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.
  *   y_bf16   device, bf16 [M][N] row-major, leading dimension N; fully overwritten.
  *   workspace, workspace_bytes   device scratch of at least tf_workspace_size(op, M, K, N)
