@@ -145,6 +145,25 @@ __device__ __forceinline__ void drain_share(uint32_t tmem_base, __nv_bfloat16* t
     }
 }
 
+// An fp16 scale has 11 significant bits, a bf16 number 8.  Rounding the scale to bf16 would put the same relative
+// error (up to 2^-8) on every weight of a group -- an error that does not average out over k.  So the scale is split
+// into its upper 8 bits and the (at most 3) bits below, both exact in bf16, and a weight is
+// fma(d, hi, d * lo): for 4-bit codes |d| <= 15 and d * lo is exact, so the result is bf16((q - z) * s) with a single
+// rounding; for 8-bit codes d * lo is rounded at 2^-9 of a term that is 2^-8 of the weight, which changes nothing.
+__device__ __forceinline__ void split_scale(float s, uint32_t& hi2, uint32_t& lo2) {
+    const uint32_t bits = __float_as_uint(s);
+    const uint32_t hi = bits & 0xFFFF0000u;                          // truncated to bf16
+    const uint32_t lo = __float_as_uint(s - __uint_as_float(hi));    // exact, at most 3 significant bits
+    hi2 = (hi >> 16) | hi;
+    lo2 = (lo >> 16) | (lo & 0xFFFF0000u);
+}
+__device__ __forceinline__ uint32_t times_scale(uint32_t d, uint32_t hi2, uint32_t lo2) {
+    uint32_t t, w;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(t) : "r"(d), "r"(lo2));
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(w) : "r"(d), "r"(hi2), "r"(t));
+    return w;
+}
+
 __device__ __forceinline__ uint32_t bf16_dup(float v) {
     const uint32_t b = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
     return b | (b << 16);
@@ -334,11 +353,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     // scales of rows (w0,g), (w0,g+8), (w0+1,g), (w0+1,g+8)
                     const uint2 sc = *(reinterpret_cast<const uint2*>(tile_smem + kWeightBytes + g * 16) + (q & 1));
                     const uint32_t sw[2] = {sc.x, sc.y};
-                    uint32_t s_g[2], s_g8[2];
+                    uint32_t s_g[2], s_g8[2], l_g[2], l_g8[2];
 #pragma unroll
                     for (int b = 0; b < 2; ++b) {
-                        s_g[b] = bf16_dup(fp16_bits_to_float((uint16_t)(sw[b] & 0xFFFFu)));
-                        s_g8[b] = bf16_dup(fp16_bits_to_float((uint16_t)(sw[b] >> 16)));
+                        split_scale(fp16_bits_to_float((uint16_t)(sw[b] & 0xFFFFu)), s_g[b], l_g[b]);
+                        split_scale(fp16_bits_to_float((uint16_t)(sw[b] >> 16)), s_g8[b], l_g8[b]);
                     }
                     if (BITS == 4) {
                         const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile_smem + kWeightBytes + kScaleBytes) + g);
@@ -355,10 +374,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                             const uint32_t xs[2] = {x.x, x.y};
 #pragma unroll
                             for (int b = 0; b < 2; ++b) {
-                                op[b][4 * i + 0] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 0), zg[b]), s_g[b]);    // row g,   k 0,1
-                                op[b][4 * i + 1] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 2), zg[b]), s_g[b]);    // row g,   k 2,3
-                                op[b][4 * i + 2] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 1), zg8[b]), s_g8[b]);  // row g+8, k 0,1
-                                op[b][4 * i + 3] = bf16x2_mul(bf16x2_sub(w4_reg_biased(xs[b], 3), zg8[b]), s_g8[b]);  // row g+8, k 2,3
+                                op[b][4 * i + 0] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 0), zg[b]), s_g[b], l_g[b]);    // row g,   k 0,1
+                                op[b][4 * i + 1] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 2), zg[b]), s_g[b], l_g[b]);    // row g,   k 2,3
+                                op[b][4 * i + 2] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 1), zg8[b]), s_g8[b], l_g8[b]);  // row g+8, k 0,1
+                                op[b][4 * i + 3] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 3), zg8[b]), s_g8[b], l_g8[b]);  // row g+8, k 2,3
                             }
                         }
                     } else {
@@ -371,10 +390,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                                 uint32_t r0, r1, r2, r3;
                                 w8_word_to_regs(xs[b][0], r0, r1);                     // (row g; k 0,1), (row g+8; k 0,1)
                                 w8_word_to_regs(xs[b][1], r2, r3);                     // (row g; k 2,3), (row g+8; k 2,3)
-                                op[b][4 * i + 0] = bf16x2_mul(r0, s_g[b]);
-                                op[b][4 * i + 1] = bf16x2_mul(r2, s_g[b]);
-                                op[b][4 * i + 2] = bf16x2_mul(r1, s_g8[b]);
-                                op[b][4 * i + 3] = bf16x2_mul(r3, s_g8[b]);
+                                op[b][4 * i + 0] = times_scale(r0, s_g[b], l_g[b]);
+                                op[b][4 * i + 1] = times_scale(r2, s_g[b], l_g[b]);
+                                op[b][4 * i + 2] = times_scale(r1, s_g8[b], l_g8[b]);
+                                op[b][4 * i + 3] = times_scale(r3, s_g8[b], l_g8[b]);
                             }
                         }
                     }

@@ -48,9 +48,16 @@ def test_unit_scales_integer_activations_are_exact(bits):
     assert np.array_equal(y, want)
 
 
+def _round_to_bf16(v: np.ndarray) -> np.ndarray:
+    """fp64 -> nearest bf16 value (8 significant bits, ties to even), returned as fp64."""
+    m, e = np.frexp(v)                       # v = m * 2^e, 0.5 <= |m| < 1
+    return np.ldexp(np.round(m * 256.0), e - 8)
+
+
 @pytest.mark.parametrize("bits", [4, 8])
 def test_one_hot_activations_pick_weights(bits):
-    """a = e_k: y[n] = bf16(bf16(q - z) * bf16(s)) -- the GEMM's documented single rounding of w."""
+    """a = e_k: y[n] is the GEMM's weight operand itself.  W4: bf16((q - z) * s), one rounding of the exact product
+    with the fp16 scale.  W8: the scale is split into its upper 8 bits and the rest, w = bf16(q * hi + bf16(q * lo))."""
     K, N = 256, 136
     p = (wl.make_w4 if bits == 4 else wl.make_w8)(1, K, N, seed=77, keep_raw=True)
     blob = torch.from_numpy(gu.pack(p)).cuda()
@@ -60,10 +67,14 @@ def test_one_hot_activations_pick_weights(bits):
         a[i, k] = 0x3F80
     y = bf16_bits_to_f64(gu.run(p, "gemm", blob_dev=blob, a_bits=a))
     qi = p.raw["q"].astype(np.float64)
+    s = np.repeat(p.scales_f16.astype(np.float64), 128, 0)
     if bits == 4:
         qi = qi - np.repeat(p.raw["z"].astype(np.float64), 128, 0)
-    s_bf = bf16_bits_to_f64(wl.f32_to_bf16_bits(p.scales_f16.astype(np.float32)))
-    w = bf16_bits_to_f64(wl.f32_to_bf16_bits((qi * np.repeat(s_bf, 128, 0)).astype(np.float32)))
+        w = _round_to_bf16(qi * s)
+    else:
+        s_hi = s.astype(np.float32).view(np.uint32) & np.uint32(0xFFFF0000)         # truncated to bf16
+        s_hi = s_hi.view(np.float32).astype(np.float64)
+        w = _round_to_bf16(qi * s_hi + _round_to_bf16(qi * (s - s_hi)))
     assert np.array_equal(y, w[ks])
 
 
