@@ -207,8 +207,9 @@ tf_status tf_gemv_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  * K, N <= 32768.  Same arguments as the GEMV.  Each packed weight tile is dequantized once
  * per CTA tile into the tensor-memory operand of the tcgen05 tensor cores as bf16 and reused by
  * every token row of the tile (the dequantize-once rule of Section 4.1); accumulation is fp32 in
- * tensor memory.  The operand is w = bf16((q-z) * bf16(s)): (q-z) exact, the fp16 scale
- * rounded to bf16, the product rounded once more (two roundings of 2^-9 relative each).
+ * tensor memory.  The operand is w = bf16((q-z) * s), the exact product rounded to bf16 once (what
+ * tf_dequant_bf16 writes); for W8 the fp16 scale is split into its upper 8 bits and the rest and
+ * w = bf16(q * hi + bf16(q * lo)), which differs from one rounding by at most 2^-17 of w.
  * Work is split evenly over the persistent CTAs in units of (output tile, 128-deep k-tile): an
  * output tile whose K range is cut between CTAs is summed in fp32 through the workspace, in CTA
  * order, by the last CTA to finish its part, so results do not depend on timing.

@@ -18,7 +18,7 @@
 //               and zeros, Section 4.2).
 //   warp 1      one thread issues tcgen05.mma (4 per k-step) and tcgen05.commit.
 //   warp 2      allocates / frees tensor memory.
-//   warps 4-11  dequantize: packed words -> (q - z) exact in bf16 -> times bf16 scale -> tcgen05.st.  The
+//   warps 4-11  dequantize: packed words -> (q - z) exact in bf16 -> times the scale, one rounding (split_scale) -> tcgen05.st.  The
 //               packed words are stored in the register order of the 16x256b store, so a word goes from
 //               shared memory to the tensor-memory operand without any shuffle.
 //   warps 12-15 epilogue: tcgen05.ld accumulator -> bf16 -> y.
