@@ -59,6 +59,7 @@ typedef enum tf_op {
 #define TF_MAX_M_GEMM   4096
 #define TF_TILE_K       128     /* k-extent of one packed tile = the AWQ group size */
 #define TF_TILE_N       64      /* n-extent of one packed tile (a "strip" of columns) */
+#define TF_WORKSPACE_HEAD_BYTES 20480   /* start of a workspace that must be zero before its first use */
 
 /*
  * The packed blob (output of tf_pack_awq / tf_pack_w8).
@@ -172,15 +173,19 @@ tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int
  *            as constants: the kernels start fetching them before the stream's earlier kernels have finished
  *            where those release their dependents early (programmatic dependent launch, as this library's
  *            own kernels do).  Ordinary stream order covers a blob written by a copy or by a kernel that does
- *            not do that; activations, results and the workspace are always touched in stream order.
+ *            not do that.  Activations, results and the workspace are always touched in stream order: every
+ *            warp that reads a_bf16, writes y_bf16 or uses the workspace first waits until all earlier work
+ *            of the stream has completed, so a call may consume what the call before it wrote.
  *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.
  *   y_bf16   device, bf16 [M][N] row-major, leading dimension N; fully overwritten.
  *   workspace, workspace_bytes   device scratch of at least tf_workspace_size(op, M, K, N)
- *            bytes.  Its first 4096 bytes must be zero before the first call that uses it; every
- *            call leaves them zero again unless it reports an error there.  Bytes [0,16) hold the
- *            device status word read by tf_device_status; the rest holds arrival counters and the
- *            fp32 partial sums of the few column strips that are split between two CTAs.  Use one
- *            workspace per stream: calls that run concurrently must not share one.
+ *            bytes.  Its first TF_WORKSPACE_HEAD_BYTES bytes must be zero before the first call that
+ *            uses it; every call leaves them zero again unless it reports an error there.  Bytes [0,16)
+ *            hold the device status word read by tf_device_status; the rest holds arrival counters and
+ *            the fp32 partial sums of the few column strips that are split between two CTAs.  GEMV and
+ *            GEMM calls lay the workspace out compatibly: one workspace of the largest size needed may
+ *            serve every call of a stream, in any order.  Use one workspace per stream: calls that run
+ *            concurrently must not share one.
  * Arithmetic: weights are kept exact ((q - z) as small integers, scale applied in fp32 to
  * per-group partial sums), fp32 accumulation, one round-to-nearest-even to bf16 at the end.
  * tf_gemv_w8a16 with M <= 2 forms the products in integers: per token and 128-deep k-tile the
@@ -214,9 +219,10 @@ tf_status tf_gemv_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  * output tile whose K range is cut between CTAs is summed in fp32 through the workspace, in CTA
  * order, by the last CTA to finish its part, so results do not depend on timing.
  * Workspace: tf_workspace_size() bytes (tens of MB: two fp32 tile slots per CTA).  Its first
- * 20480 bytes (status word and arrival counters) must be zero before the first call that uses
- * it; every call leaves them zero again unless it reports an error there.  One workspace per
- * stream: calls that run concurrently must not share one.
+ * TF_WORKSPACE_HEAD_BYTES bytes (status word and arrival counters) must be zero before the first
+ * call that uses it; every call leaves them zero again unless it reports an error there.  One
+ * workspace per stream (it may be the one the GEMV calls of that stream use): calls that run
+ * concurrently must not share one.
  * Errors as for the GEMV; M range 1..4096.
  */
 tf_status tf_gemm_w4a16(const void* packed, const void* a_bf16, void* y_bf16,
@@ -232,7 +238,7 @@ tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  * plug-in in a process whose memory pool another framework owns, a thread that must stay out of the
  * allocator, code inside a stream capture.)
  *   Scratch (arrival counters, fp32 partial sums of strips cut between two CTAs, status word) is a fixed
- *   array of about 1.26 MB inside the library's device image: every GPU that loads the library holds it
+ *   array of about 1.27 MB inside the library's device image: every GPU that loads the library holds it
  *   until the process exits.  It covers every shape tf_gemv_w4a16 accepts (1 <= M <= 16, K and N up to
  *   32768) on devices with any SM count (at most 160 persistent CTAs are used); shapes beyond those limits
  *   are rejected with TF_ERR_SHAPE.
@@ -271,6 +277,17 @@ tf_status tf_gemv_awq_raw(const uint32_t* qweight, const uint16_t* scales_fp16, 
 /* Scratch bytes tf_gemv_awq_raw needs on the current device (0 if the shape is illegal or the device is
  * not compute capability 10.x). */
 size_t tf_gemv_awq_raw_workspace_size(int M, int K, int N, int group_size);
+
+/*
+ * Test and tuning hook: the launch geometry tf_gemv_w4a16 / tf_gemv_w8a16 would choose for this shape (Section
+ * 4.4 maps work to cores statically; here the mapping depends on the shape, and tests assert which one they hit).
+ *   sm_count  SMs to plan for; <= 0 = the current device (then TF_ERR_ARCH / TF_ERR_CUDA as for a compute call).
+ *   out       host, 8 ints: persistent CTAs, threads per CTA, consumer warps, ring stages, whole-SM CTA (1) or
+ *             half-SM (0), integer path (1/0), CTAs per cluster (1 = cut strips go through the workspace), and
+ *             the number of clusters (cluster mode) or of CTAs that get tiles (otherwise).
+ * Pure host code apart from the device query; launches nothing.  Errors: TF_ERR_NULL, TF_ERR_SHAPE.
+ */
+tf_status tf_gemv_plan(int bits, int M, int K, int N, int sm_count, int* out);
 
 /* Scratch bytes the given operation needs for this shape (0 if none; 0 also if the shape
  * is illegal -- the compute call then reports TF_ERR_SHAPE). */

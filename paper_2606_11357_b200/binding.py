@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIG
 EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
-           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size")
+           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan")
 
 
 class TileFuseError(RuntimeError):
@@ -55,6 +55,7 @@ def lib() -> ctypes.CDLL:
         L.tf_gemv_w4a16_static.restype = c_int
         L.tf_gemv_w4a16_static.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_workspace_size.restype, L.tf_workspace_size.argtypes = c_size, [c_int] * 4
+        L.tf_gemv_plan.restype, L.tf_gemv_plan.argtypes = c_int, [c_int] * 5 + [vp]
         L.tf_dequant_bf16.restype, L.tf_dequant_bf16.argtypes = c_int, [vp, vp, c_int, c_int, c_int, vp]
         L.tf_gemv_awq_raw.restype = c_int
         L.tf_gemv_awq_raw.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, c_int, vp, c_size, vp]
@@ -133,6 +134,14 @@ def tf_pack_concat(parts, out=None) -> np.ndarray:
     ptrs = (ctypes.c_void_p * max(len(parts), 1))(*[p.ctypes.data for p in parts])
     _check("tf_pack_concat", lib().tf_pack_concat(ctypes.cast(ptrs, ctypes.c_void_p), len(parts), out.ctypes.data, out.nbytes))
     return out
+
+
+def tf_gemv_plan(bits: int, M: int, K: int, N: int, sm_count: int = 0) -> dict:
+    """Launch geometry the GEMV would choose (sm_count <= 0: the current device)."""
+    out = (ctypes.c_int * 8)()
+    _check("tf_gemv_plan", lib().tf_gemv_plan(bits, M, K, N, sm_count, ctypes.cast(out, ctypes.c_void_p)))
+    names = ("grid", "threads", "consumers", "stages", "full", "i8", "cluster", "nclusters")
+    return dict(zip(names, (int(v) for v in out)))
 
 
 def tf_workspace_size(op: int, M: int, K: int, N: int) -> int:

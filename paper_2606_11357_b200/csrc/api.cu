@@ -97,6 +97,23 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_w8a16(const 
     return gemm(8, packed, a, y, M, K, N, workspace, workspace_bytes, stream);
 }
 
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_plan(int bits, int M, int K, int N, int sm_count, int* out) {
+    if (!out) return TF_ERR_NULL;
+    if (bits != 4 && bits != 8) return TF_ERR_SHAPE;
+    if (M < 1 || M > TF_MAX_M_GEMV || tf_packed_size(bits, K, N, tf::kTileK) == 0) return TF_ERR_SHAPE;
+    if (sm_count <= 0) {
+        DeviceInfo dev;
+        tf_status st = device_info(&dev);
+        if (st != TF_OK) return st;
+        sm_count = dev.sm_count;
+    }
+    if (sm_count > tf::kGemvMaxGrid) sm_count = tf::kGemvMaxGrid;
+    const tf::GemvPlan p = tf::plan_gemv(bits, M, K, N, sm_count);
+    out[0] = p.grid; out[1] = p.threads; out[2] = p.consumers; out[3] = p.stages;
+    out[4] = p.full ? 1 : 0; out[5] = p.i8 ? 1 : 0; out[6] = p.cluster; out[7] = p.nclusters;
+    return TF_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) size_t tf_workspace_size(int op, int M, int K, int N) {
     const int bits = (op == TF_OP_GEMV_W4A16 || op == TF_OP_GEMM_W4A16) ? 4 : 8;
     if (op < TF_OP_GEMV_W4A16 || op > TF_OP_GEMM_W8A16) return 0;

@@ -11,13 +11,15 @@
 //                   instruction of this warp competes for issue slots with consumer warps that never idle.
 //                   It reads nothing but weights, which are constants, so it does not wait for earlier
 //                   kernels of the stream.
-//   consumer warps: take tiles round-robin.  A warp first asks for the tile's activations -- its own MMA
+//   consumer warps: take tiles round-robin.  A warp reads the activations of a tile -- its own MMA
 //                   fragment, 8 bytes per lane and 16-k block (integer path: its 4 k of the tile's 128 per
-//                   token), straight from global memory (they sit in
-//                   L2) -- and only then waits for the tile's weights, so the two latencies overlap and the
-//                   ring holds nothing but weights (staging activations through the ring put a TMA load
-//                   behind the dependency wait of every call, about 1 us, and took ring space from the
-//                   weights: half of it for 9..16 tokens).  128-bit shared loads, codes -> exact small-integer bf16
+//                   token) -- straight from global memory (they sit in L2), never before the kernels ahead
+//                   of this one on the stream have completed (every consumer warp executes the dependency
+//                   wait first), and one tile ahead: the registers of a k-block are refilled for the warp's
+//                   next tile as soon as that k-block's MMAs have been issued, so the L2 latency runs under
+//                   the rest of the tile.  The ring holds nothing but weights (staging activations through
+//                   the ring put a TMA load behind the dependency wait of every call, about 1 us, and took
+//                   ring space from the weights: half of it for 9..16 tokens).  128-bit shared loads, codes -> exact small-integer bf16
 //                   (q - z), contraction with the activations on the warp-level tensor-core MMA
 //                   (weights = the 16x16 operand, up to 8 tokens = the 16x8 operand: the per-weight
 //                   cost does not grow with M), fp16 scale applied in fp32 once per group.
@@ -183,9 +185,10 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     }
     __syncthreads();
     // Programmatic dependent launch: the next kernel on the stream may start as SMs free up.  In this kernel
-    // only the packed weights (constants) are read before grid_dependency_wait(); activations, y and the
-    // workspace are touched after it.  (What keeps two half-SM CTAs of one GEMV off the same SM when they come in
-    // behind a whole-SM kernel is decided at launch: see launch_one.)
+    // only the packed weights (constants) are read before grid_dependency_wait(): the producer lane never waits,
+    // every consumer warp waits before its first activation load, the reducer warp before it touches y or the
+    // workspace, thread 0 before it writes the status word.  (What keeps two half-SM CTAs of one GEMV off the same
+    // SM when they come in behind a whole-SM kernel is decided at launch: see launch_one.)
     grid_launch_dependents();
 
     if (warp == 0) {
@@ -350,6 +353,45 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 
         int i = 0, sidx = 0, chunk_base = 0;
         int cg_cur = 0, s_cur = 0, use_cur = 0;         // this warp's position in the ring (chunks only move forward)
+        // This warp's tiles are the local indices cw, cw + nconsumers, ... of the CTA's range, whatever strip they
+        // fall into.  The activations of a tile are this lane's own MMA fragments (integer path: its 4 k per token),
+        // read straight from global memory.  They are written by earlier kernels of the stream, so nothing is read
+        // before the dependency wait; the fragments of the NEXT tile are then requested as soon as a k-block of the
+        // current tile has used its registers, so their L2 latency runs under the rest of the tile.
+        uint2 araw[2];                                  // integer path: token m, k = 128 T + 4 lane .. +3
+        uint2 ag[!I8 ? MT : 1][!I8 ? 8 : 1];            // token g (+8): k = 128 T + 16 kb + 4t .. +3
+        auto act_tile_base = [&](int local_tile) -> const __nv_bfloat16* {
+            const int tile_abs = t0 + local_tile;
+            return a_glob + (size_t)(tile_abs - (tile_abs / ktiles) * ktiles) * kTileK;
+        };
+        auto load_araw = [&](const __nv_bfloat16* base) {
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                araw[m] = make_uint2(0u, 0u);
+                if (m < M) araw[m] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)m * K + 4 * lane));
+            }
+        };
+        auto load_ag_kb = [&](const __nv_bfloat16* base, int kb) {
+#pragma unroll
+            for (int mt = 0; mt < (!I8 ? MT : 1); ++mt)
+                if (g + 8 * mt < M)
+                    ag[mt][!I8 ? kb : 0] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)(g + 8 * mt) * K + 4 * t + 16 * kb));
+        };
+        grid_dependency_wait();                         // the activations belong to earlier kernels until now
+        if constexpr (!I8) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int kb = 0; kb < 8; ++kb) ag[mt][kb] = make_uint2(0u, 0u);
+        }
+        if (cw < ntiles) {
+            const __nv_bfloat16* base = act_tile_base(cw);
+            if constexpr (I8) load_araw(base);
+            else {
+#pragma unroll
+                for (int kb = 0; kb < 8; ++kb) load_ag_kb(base, kb);
+            }
+        }
         while (i < ntiles && !aborted) {
             const int tile0 = t0 + i;
             const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
@@ -372,26 +414,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 cg_cur = cg;
                 while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
                 const int s = s_cur;
-                uint2 araw[2];                                  // integer path: token m, k = 128 T + 4 lane .. +3
-                if constexpr (I8) {
-#pragma unroll
-                    for (int m = 0; m < 2; ++m) {
-                        araw[m] = make_uint2(0u, 0u);
-                        if (m < M) araw[m] = __ldg(reinterpret_cast<const uint2*>(a_glob + (size_t)m * K + (size_t)(T0 + lj) * kTileK + 4 * lane));
-                    }
-                }
-                uint2 ag[!I8 ? MT : 1][!I8 ? 8 : 1];            // token g (+8): k = 128 T + 16 kb + 4t .. +3
-                if constexpr (!I8) {
-                    const __nv_bfloat16* arow = a_glob + (size_t)(T0 + lj) * kTileK + 4 * t;
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                        for (int kb = 0; kb < 8; ++kb) {
-                            ag[mt][kb] = make_uint2(0u, 0u);
-                            if (g + 8 * mt < M)
-                                ag[mt][kb] = __ldg(reinterpret_cast<const uint2*>(arow + (size_t)(g + 8 * mt) * K + 16 * kb));
-                        }
-                }
+                const bool has_next = j + nconsumers < ntiles;
+                const __nv_bfloat16* next_base = act_tile_base(has_next ? j + nconsumers : j);
                 if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
                     const long long t_begin = clock64();
                     while (stage_tag[s] != (uint32_t)cg && !aborted) {
@@ -452,6 +476,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                             }
                         }
                     }
+                    if (has_next) load_araw(next_base);                 // the next tile's activations, under this tile's MMAs
                     if (lane == 0) {                                    // columns without a token contribute nothing
 #pragma unroll
                         for (int c = 3; c < 8; ++c)
@@ -552,6 +577,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                         for (int mt = 0; mt < MT; ++mt)
                             mma_bf16_16816(gacc[w][mt], r0, r1, r2, r3, av[mt].x, av[mt].y);
                     }
+                    if (has_next) load_ag_kb(next_base, kb);    // this k-block's registers are free: ask for the next tile's
                 }
                 // all shared-memory reads of this tile are done: hand its share of the stage back to the
                 // producer (the last tile of a short chunk also returns the shares of the missing tiles)

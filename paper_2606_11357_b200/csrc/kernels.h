@@ -36,14 +36,19 @@ constexpr int kGemvStageBytes = 17408;        // 17 x 1024 >= 4 x 4256 and >= 2 
 constexpr int kGemvMaxM = 16;
 constexpr int kGemvI8MaxM = 2;                // int8 weights, up to this many tokens: the GEMV runs on the integer warp MMA
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
-// Workspace layout: [0,16) status word | [256, 256+4*512) per-strip arrival counters | partial sums
+// Workspace layout, shared with the GEMM so that one workspace serves every call of a stream:
+//   [0,16) status word | [256, 256+4*512) GEMV per-strip arrival counters | [4096, 20480) GEMM per-tile arrival
+//   counters | from 20480: partial sums (written before they are read, so either kernel may leave anything there).
+// Everything below kWorkspaceHeadBytes is zero between calls.
+constexpr int kWorkspaceHeadBytes = 20480;
 constexpr int kGemvCounterOffset = 256;
-constexpr int kGemvPartialOffset = 4096;
+constexpr int kGemvCounterEnd = 4096;         // the GEMV touches no counter beyond this
+constexpr int kGemvPartialOffset = kWorkspaceHeadBytes;
 constexpr size_t kGemvWorkspaceBytes = kGemvPartialOffset + (size_t)kGemvMaxGrid * 2 * kGemvMaxM * 64 * 4;
 
 struct GemvPlan {
     int grid;          // persistent CTAs
-    int threads;       // 32 * (consumers + 1)
+    int threads;       // 32 * (consumers + 2): producer warp, reducer warp, consumer warps
     int consumers;     // consumer warps
     int stages;        // ring depth
     bool full;         // whole-SM configuration
@@ -73,7 +78,7 @@ cudaError_t launch_dequant(int bits, const void* blob, void* w_bf16, int K, int 
 
 // Fused W4A16 GEMV on the AWQ arrays as they come (no pre-tiling): the second arm of the layout ablation.
 struct RawGemvPlan {
-    bool mma;            // 3..16 tokens: tensor-core kernel (units are 16-row blocks); else the fp32 kernel (units are groups)
+    bool mma;            // 9..16 tokens: tensor-core kernel (units are 16-row blocks); up to 8: the fp32 kernel (units are groups)
     int groups;          // units along K
     int col_blocks;      // blocks of 256 (fp32) or 64 (tensor-core) output columns
     int splits;          // CTAs that share a column block (split-K over whole units)

@@ -8,7 +8,7 @@
 // no cudaMalloc / cudaFree and no library routine that allocates.
 //
 // The array exists once per GPU that loads the library and stays until the process exits
-// (kStaticScratchBytes, about 1.26 MB).  All calls share it and it keeps whatever the last call left: the
+// (kStaticScratchBytes, about 1.27 MB).  All calls share it and it keeps whatever the last call left: the
 // bytes that must start at zero are cleared on the stream before every launch, and two calls that overlap
 // on the GPU (different streams, or graphs run concurrently) would race on it -- serialise them.
 #include <cuda_runtime.h>
@@ -78,7 +78,7 @@ tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_b
     if (st != TF_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // status word and arrival counters must start at zero; the partial sums are always written before read
-    if (cudaMemsetAsync(dev->scratch, 0, tf::kGemvPartialOffset, stream) != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    if (cudaMemsetAsync(dev->scratch, 0, tf::kGemvCounterEnd, stream) != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
     const int ctas = dev->sm_count < kStaticMaxGrid ? dev->sm_count : kStaticMaxGrid;
     const tf::GemvPlan plan = tf::plan_gemv(4, M, K, N, ctas);
     if (tf::launch_gemv(4, plan, packed, a_bf16, y_bf16, M, K, N, dev->scratch, stream) != cudaSuccess) {

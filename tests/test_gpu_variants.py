@@ -56,8 +56,8 @@ def test_illegal_group_sizes_are_rejected():
     assert tf.tf_packed_size(8, 1024, 64, 1024) > 0
 
 
-@pytest.mark.parametrize("kind,M,K,N,zero_bytes", [("gemv", 1, 4096, 1024, 4096), ("gemv", 16, 4096, 4096, 4096),
-                                                   ("gemv", 4, 1536, 328, 4096), ("gemm", 300, 2048, 1096, 20480),
+@pytest.mark.parametrize("kind,M,K,N,zero_bytes", [("gemv", 1, 4096, 1024, 20480), ("gemv", 16, 4096, 4096, 20480),
+                                                   ("gemv", 4, 1536, 328, 20480), ("gemm", 300, 2048, 1096, 20480),
                                                    ("gemm", 512, 4096, 640, 20480)])
 def test_workspace_head_is_left_zero(kind, M, K, N, zero_bytes):
     """The status word and the arrival counters must be zero again after a call, so the same workspace serves
@@ -205,3 +205,29 @@ def test_gemv_on_two_streams_with_their_own_workspaces():
     for i, p in enumerate(probs):
         gu.check_against_oracle(p, gu.bits_of(ys[0][i]))
         assert np.array_equal(gu.bits_of(ys[0][i]), gu.bits_of(ys[1][i]))      # same inputs, bit-identical outputs
+
+
+def test_gemv_and_gemm_share_one_workspace():
+    """One workspace of the largest size serves every call of a stream, in any order: the GEMV's partial sums of cut
+    strips and the GEMM's arrival counters must not use the same bytes, and both leave the head of it zero."""
+    Mv, Mm, K, N = 4, 160, 4096, 4096                       # both shapes cut strips / tiles between CTAs
+    pv = wl.make_w4(Mv, K, N, seed=1201)
+    pm = wl.make_w4(Mm, K, N, seed=1202)
+    bv, bm = torch.from_numpy(gu.pack(pv)).cuda(), torch.from_numpy(gu.pack(pm)).cuda()
+    av, am = gu.to_device_bf16(pv.a_bf16), gu.to_device_bf16(pm.a_bf16)
+    yv = torch.empty((Mv, N), dtype=torch.bfloat16, device="cuda")
+    ym = torch.empty((Mm, N), dtype=torch.bfloat16, device="cuda")
+    need = max(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, Mv, K, N), tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, Mm, K, N))
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    for order in ("vm", "mv", "vvm", "mmv"):
+        yv.fill_(float("nan"))
+        ym.fill_(float("nan"))
+        for op in order:
+            if op == "v":
+                tf.tf_gemv_w4a16(bv, av, yv, Mv, K, N, ws)
+            else:
+                tf.tf_gemm_w4a16(bm, am, ym, Mm, K, N, ws)
+        assert tf.tf_device_status(ws) == 0
+        assert int(ws[:20480].to(torch.int32).sum().item()) == 0
+        gu.check_against_oracle(pv, gu.bits_of(yv))
+        gu.check_against_oracle(pm, gu.bits_of(ym))

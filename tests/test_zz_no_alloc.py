@@ -55,3 +55,37 @@ def test_static_scratch_gemv_rejects_out_of_range():
     assert L.tf_gemv_w4a16_static(ok, ok, ok, 1, 32768 + 128, 8, None) == 2    # K beyond the maximum
     assert L.tf_gemv_w4a16_static(ok, ok, ok, 1, 128, 32768 + 8, None) == 2    # N beyond the maximum
     assert L.tf_gemv_w4a16_static(ok, ctypes.c_void_p(0x1008), ok, 1, 128, 8, None) == 3
+
+
+def test_static_scratch_gemv_chain_consumes_previous_output():
+    """Two static calls back to back where the second multiplies what the first writes (no host synchronisation in
+    between, intermediate pre-filled with NaN on the stream): same bits as the workspace path, within the
+    oracle's tolerance."""
+    import copy
+    M = 4
+    p1 = wl.make_w4(M, 4096, 14336, seed=103)
+    p2 = wl.make_w4(M, 14336, 4096, seed=104)
+    b1, b2 = torch.from_numpy(gu.pack(p1)).cuda(), torch.from_numpy(gu.pack(p2)).cuda()
+    a0 = gu.to_device_bf16(p1.a_bf16)
+    y1 = torch.empty((M, 14336), dtype=torch.bfloat16, device="cuda")
+    y2 = torch.empty((M, 4096), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, M, 4096, 4096), dtype=torch.uint8, device="cuda")
+    results = []
+    for static in (False, True, True):
+        y1.fill_(float("nan"))
+        y2.fill_(float("nan"))
+        if static:
+            tf.tf_gemv_w4a16_static(b1, a0, y1, M, 4096, 14336)
+            tf.tf_gemv_w4a16_static(b2, y1, y2, M, 14336, 4096)
+        else:
+            tf.tf_gemv_w4a16(b1, a0, y1, M, 4096, 14336, ws)
+            tf.tf_gemv_w4a16(b2, y1, y2, M, 14336, 4096, ws)
+        torch.cuda.synchronize()
+        results.append((gu.bits_of(y1), gu.bits_of(y2)))
+    assert tf.tf_device_status(ws) == 0
+    for o1, o2 in results[1:]:
+        assert np.array_equal(o1, results[0][0]) and np.array_equal(o2, results[0][1])
+    gu.check_against_oracle(p1, results[1][0])
+    q2 = copy.copy(p2)
+    q2.a_bf16 = results[1][0]
+    gu.check_against_oracle(q2, results[1][1])
