@@ -188,11 +188,13 @@ tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int
  *            concurrently must not share one.
  * Arithmetic: weights are kept exact ((q - z) as small integers, scale applied in fp32 to
  * per-group partial sums), fp32 accumulation, one round-to-nearest-even to bf16 at the end.
- * tf_gemv_w8a16 with M <= 2 forms the products in integers: per token and 128-deep k-tile the
+ * With M <= 2 both calls form the products in integers: per token and 128-deep k-tile the
  * activations are rewritten on the tile's own power-of-two scale (exact for values within 2^14
- * of the tile's largest magnitude, rounded at 2^-22 of it below that), multiplied with the int8
- * codes exactly in 32 bits, and scaled back in fp32.  An Inf or NaN activation makes every output
- * of its token NaN there (the floating-point paths give Inf or NaN, as IEEE arithmetic does).
+ * of the tile's largest magnitude, rounded at 2^-22 of it below that), multiplied with the codes
+ * exactly in 32 bits (4-bit: sum of q times activation minus z times the sum of the activations,
+ * both exact integers, so q == z still gives exactly 0), and scaled back in fp32.  An Inf or NaN
+ * activation makes every output of its token NaN there (the floating-point paths give Inf or NaN,
+ * as IEEE arithmetic does).
  * Each persistent CTA streams one contiguous range of packed tiles; a strip of 64 output
  * columns that is cut between CTAs is summed in CTA order by the last CTA to finish it.
  * The blob must be at least tf_packed_size(bits, K, N, 128) bytes for the K, N passed here.

@@ -44,6 +44,7 @@
 
 namespace tf {
 
+
 namespace {
 
 // Integer warp MMA: D(16x8, s32) += A(16x32, s8) . B(32x8, s8).  Thread (g, t): a0 = row g, k 4t..4t+3; a1 = row g+8;
@@ -56,6 +57,17 @@ __device__ __forceinline__ void mma_s8_16832(int d[4], uint32_t a0, uint32_t a1,
 __device__ __forceinline__ void mma_s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
     const int zero = 0;
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
+}
+
+// The same shapes with unsigned bytes in the 16-row operand (4-bit codes 0..15 as they come out of a packed word).
+__device__ __forceinline__ void mma_u8s8_16832(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_u8s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    const int zero = 0;
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
                  : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
 }
 
@@ -356,14 +368,11 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         // This warp's tiles are the local indices cw, cw + nconsumers, ... of the CTA's range, whatever strip they
         // fall into.  The activations of a tile are this lane's own MMA fragments (integer path: its 4 k per token),
         // read straight from global memory.  They are written by earlier kernels of the stream, so nothing is read
-        // before the dependency wait; the fragments of the NEXT tile are then requested as soon as a k-block of the
-        // current tile has used its registers, so their L2 latency runs under the rest of the tile.
+        // before the dependency wait; up to 8 tokens the fragments of the NEXT tile are then requested as soon as a
+        // k-block of the current tile has used its registers, so their L2 latency runs under the rest of the tile.
         uint2 araw[2];                                  // integer path: token m, k = 128 T + 4 lane .. +3
         uint2 ag[!I8 ? MT : 1][!I8 ? 8 : 1];            // token g (+8): k = 128 T + 16 kb + 4t .. +3
-        auto act_tile_base = [&](int local_tile) -> const __nv_bfloat16* {
-            const int tile_abs = t0 + local_tile;
-            return a_glob + (size_t)(tile_abs - (tile_abs / ktiles) * ktiles) * kTileK;
-        };
+        int T_act = (t0 + cw) % ktiles;                 // k-tile index of this warp's current tile (one division per kernel)
         auto load_araw = [&](const __nv_bfloat16* base) {
 #pragma unroll
             for (int m = 0; m < 2; ++m) {
@@ -384,8 +393,12 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 #pragma unroll
                 for (int kb = 0; kb < 8; ++kb) ag[mt][kb] = make_uint2(0u, 0u);
         }
-        if (cw < ntiles) {
-            const __nv_bfloat16* base = act_tile_base(cw);
+        // One tile ahead only for up to 8 tokens: with 16 tokens the fragments are 32 registers that would stay live
+        // across the whole tile, and the kernel is slower with them (measured: 62.1 against 55.7 us over the four
+        // layer shapes); there a tile's activations are requested when the tile begins, before the wait for its weights.
+        constexpr bool kAhead = MT == 1;
+        if (kAhead && cw < ntiles) {
+            const __nv_bfloat16* base = a_glob + (size_t)T_act * kTileK;
             if constexpr (I8) load_araw(base);
             else {
 #pragma unroll
@@ -414,8 +427,16 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 cg_cur = cg;
                 while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
                 const int s = s_cur;
-                const bool has_next = j + nconsumers < ntiles;
-                const __nv_bfloat16* next_base = act_tile_base(has_next ? j + nconsumers : j);
+                const bool has_next = kAhead && j + nconsumers < ntiles;
+                if constexpr (!kAhead) {
+                    const __nv_bfloat16* base = a_glob + (size_t)T_act * kTileK;
+#pragma unroll
+                    for (int kb = 0; kb < 8; ++kb) load_ag_kb(base, kb);
+                }
+                int T_nx = T_act + nconsumers;                  // the warp's next tile is nconsumers tiles further along K
+                while (T_nx >= ktiles) T_nx -= ktiles;
+                T_act = T_nx;
+                const __nv_bfloat16* next_base = a_glob + (size_t)T_nx * kTileK;
                 if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
                     const long long t_begin = clock64();
                     while (stage_tag[s] != (uint32_t)cg && !aborted) {
@@ -430,15 +451,18 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 
                 const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
                 if constexpr (I8) {
-                    // ---- integer path (int8 weights, 1 or 2 tokens): codes x activation pieces on the integer warp MMA ----
+                    // ---- integer path (1 or 2 tokens): codes x activation pieces on the integer warp MMA ----
                     // The 128 activations of a (token, k-tile) are scaled by 2^(148 - emax) (emax = largest biased
                     // exponent among them), rounded to integers |v| < 2^22 and split into signed bytes
                     // v = p0 + 256 p1 + 65536 p2: values within 2^14 of the largest are exact, smaller ones are rounded
-                    // at 2^-22 of it.  Piece j of token m is column 3m + j of the MMA's 8-column operand; the int8 codes
-                    // are the other operand as they are, so no weight is ever converted:
+                    // at 2^-22 of it.  Piece j of token m is column 3m + j of the MMA's 8-column operand; the codes are
+                    // the other operand as they are (int8), or after one AND and one shift + AND per packed word (4-bit:
+                    // the low nibbles of a word are this lane's row g, the high nibbles its row g + 8, as unsigned bytes),
+                    // so no weight is ever converted to floating point:
                     //     D[n][3m+j] = sum_k q[k][n] p_j[m][k]            (exact, 32-bit integers)
+                    //     4-bit: D[n][3m+j] -= z[n] sum_k p_j[m][k]       (the zero point of Eq. 2, still exact)
                     //     y[m][n] += s[n] 2^(emax-148) sum_j 256^j D[n][3m+j]
-                    static_assert(!I8 || (BITS == 8 && MT == 1), "the integer path is built for int8 weights and up to 2 tokens");
+                    static_assert(!I8 || MT == 1, "the integer path is built for up to 2 tokens");
                     uint32_t* scr = pscr + cw * 256;                    // [column][36 words]: word of lane L at (L&3)*8 + (L>>2)
                     // [column]: 2^(emax-148) 256^j in 8-byte entries behind the 6 x 36 words, a thread's two columns = one 16-byte load
                     // (with 4-byte entries and an 8-byte load the same kernel ran 12 % slower: measured, cause not established)
@@ -459,20 +483,23 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                             v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
                             v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
                             v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
-                            // 4 x 3 byte transpose: one word per piece, bytes in k order
+                            // 4 x 3 byte transpose: one word per piece, bytes in the k order of the weight operand's bytes
+                            // (int8: k, k+1, k+2, k+3; 4-bit: k, k+2, k+1, k+3, the order of a packed word's nibble pairs)
                             const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
                             const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
                             uint32_t word[3];
-                            word[0] = __byte_perm(ab01, cd01, 0x5410) ^ 0x80808080u;
-                            word[1] = __byte_perm(ab01, cd01, 0x7632) ^ 0x80808080u;
-                            word[2] = __byte_perm(ab2, cd2, 0x5410) ^ 0x80808080u;
+                            word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+                            word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
+                            word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
                             // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
                             const float se = e == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((e - 21u) << 23);
 #pragma unroll
                             for (int j = 0; j < 3; ++j) {
                                 const int c = 3 * m + j;
                                 scr[c * 36 + (lane & 3) * 8 + (lane >> 2)] = word[j];
-                                if (lane == 0) col_meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), 0u);
+                                int psum = 0;                           // 4-bit: sum of the piece over the tile's 128 k, for the zero point
+                                if constexpr (BITS == 4) psum = __reduce_add_sync(0xFFFFFFFFu, __dp4a((int)word[j], 0x01010101, 0));
+                                if (lane == 0) col_meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum);
                             }
                         }
                     }
@@ -496,6 +523,22 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     }
                     __syncwarp();                                       // the scratch is rewritten for the next tile
                     int d[4][4];
+                    if constexpr (BITS == 4) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {                   // 32 k per MMA: k-blocks 2i and 2i+1, one packed word each
+                            const uint4 v0 = *reinterpret_cast<const uint4*>(tile + ((size_t)(2 * i) * 32 + lane) * 16);
+                            const uint4 v1 = *reinterpret_cast<const uint4*>(tile + ((size_t)(2 * i + 1) * 32 + lane) * 16);
+#pragma unroll
+                            for (int w = 0; w < 4; ++w) {
+                                const uint32_t x0 = w == 0 ? v0.x : w == 1 ? v0.y : w == 2 ? v0.z : v0.w;
+                                const uint32_t x1 = w == 0 ? v1.x : w == 1 ? v1.y : w == 2 ? v1.z : v1.w;
+                                const uint32_t a0 = x0 & 0x0F0F0F0Fu, a1 = (x0 >> 4) & 0x0F0F0F0Fu;     // rows g, g + 8: k-block 2i
+                                const uint32_t a2 = x1 & 0x0F0F0F0Fu, a3 = (x1 >> 4) & 0x0F0F0F0Fu;     // k-block 2i + 1
+                                if (i == 0) mma_u8s8_16832_first(d[w], a0, a1, a2, a3, bw[0], bw[1]);
+                                else mma_u8s8_16832(d[w], a0, a1, a2, a3, bw[2 * i], bw[2 * i + 1]);
+                            }
+                        }
+                    } else {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {                       // 32 k per MMA: k-blocks 2i and 2i+1
                         uint4 wv[2][2];
@@ -516,6 +559,18 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                             }
                             if (i == 0) mma_s8_16832_first(d[w], a[0], a[1], a[2], a[3], bw[0], bw[1]);
                             else mma_s8_16832(d[w], a[0], a[1], a[2], a[3], bw[2 * i], bw[2 * i + 1]);
+                        }
+                    }
+                    }
+                    if constexpr (BITS == 4) {
+                        // zero point: every code of row n stands for q - z[n], so the row's sum loses z[n] times the column's piece sum
+                        const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile + kWeightBytes + kScaleBytes) + g);
+                        const int p0 = (int)cm.y, p1 = (int)cm.w;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            const int zr = (int)((zword >> (4 * w)) & 15u), zr8 = (int)((zword >> (4 * w + 16)) & 15u);
+                            d[w][0] -= zr * p0; d[w][1] -= zr * p1;
+                            d[w][2] -= zr8 * p0; d[w][3] -= zr8 * p1;
                         }
                     }
                     __syncwarp();
@@ -789,7 +844,8 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     // launch next to a plain one does not (about 2.7 us per transition, measured), and in a pass over layers of
     // different sizes that loss is larger than what the short hand-over wins for up to 8 tokens.
     const int one_round = gemv_max_consumers(mt, mt == 2);
-    if (p.cluster > 1 && mt == 2 && tiles_per_cta <= 16 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
+    const bool cluster_ok = mt == 2;
+    if (p.cluster > 1 && cluster_ok && tiles_per_cta <= 16 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
         p.grid = p.nclusters * p.cluster;
         tiles_per_cta = best_t;
     } else {
@@ -797,11 +853,13 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
         p.nclusters = active;
         if (mt == 1 && p.grid < sm_count) p.grid = sm_count;
     }
-    // Long ranges amortise the start of the kernel: take the whole SM (more consumer warps, deeper ring).  Short
-    // ones gain more from the next GEMV's CTAs sitting beside this one's with their rings already full.
-    const bool i8_path = bits == 8 && M <= kGemvI8MaxM;
-    p.full = mt == 2 || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= (i8_path ? kGemvFullFromBytesI8 : kGemvFullFromBytes);
-    p.i8 = bits == 8 && M <= kGemvI8MaxM && p.cluster == 1;
+    // The floating-point path is bound by instruction issue in its consumer warps: it takes the whole SM (12 consumer
+    // warps, deeper ring).  The integer path of 1 and 2 tokens needs a fraction of the instructions; its short ranges
+    // gain more from the next GEMV's CTAs sitting beside this one's with their rings already full, long ones
+    // amortise the start of the kernel and take the whole SM too.
+    const bool i8_path = M <= kGemvI8MaxM;
+    p.full = mt == 2 || !i8_path || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= kGemvFullFromBytesI8;
+    p.i8 = M <= kGemvI8MaxM && p.cluster == 1;
     // the integer path leaves the warps waiting for data, not for issue slots: 8 of them keep more tiles in flight
     // (4096x14336, 1 token: 13.7 us with 8 warps, 14.2 us with 12)
     p.consumers = p.i8 && p.full ? 8 : gemv_max_consumers(mt, p.full);
@@ -852,6 +910,7 @@ void note_launch(cudaStream_t stream, bool whole_sm) {
 }  // namespace
 
 void note_whole_sm_launch(cudaStream_t stream) { note_launch(stream, true); }
+
 
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
@@ -917,11 +976,9 @@ static cudaError_t launch_bits(const GemvPlan& p, const void* blob, const void* 
                       : launch_one<BITS, 1, false, true, false>(p, blob, a, y, M, K, N, workspace, stream);
     }
     if (M > 8) return launch_one<BITS, 2, true, false, false>(p, blob, a, y, M, K, N, workspace, stream);
-    if constexpr (BITS == 8) {
-        if (p.i8)
-            return p.full ? launch_one<8, 1, true, false, true>(p, blob, a, y, M, K, N, workspace, stream)
-                          : launch_one<8, 1, false, false, true>(p, blob, a, y, M, K, N, workspace, stream);
-    }
+    if (p.i8)
+        return p.full ? launch_one<BITS, 1, true, false, true>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<BITS, 1, false, false, true>(p, blob, a, y, M, K, N, workspace, stream);
     return p.full ? launch_one<BITS, 1, true, false, false>(p, blob, a, y, M, K, N, workspace, stream)
                   : launch_one<BITS, 1, false, false, false>(p, blob, a, y, M, K, N, workspace, stream);
 }

@@ -6,25 +6,27 @@
 namespace tf {
 
 // ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
-// Up to 8 tokens, short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs fit beside
-// this one's and fill their rings while it finishes.  Up to 8 tokens, long ranges: the whole SM, 12 consumer
-// warps and a ring deep enough to keep HBM busy while 12 tiles are being consumed.
-// 9..16 tokens: twice the MMA and activation work per tile and the whole SM, but 8 consumer warps: every tile a warp
-// is working on is a tile that is not in flight (measured on the four layer shapes with the ring holding weights only:
-// 8 warps 7.9 / 4.1 / 14.5 / 15.4 us, 10 warps 8.4 / 4.1 / 15.2 / 16.1 us; 12 warps do not fit the register file).
+// Three configurations, chosen by plan_gemv:
+//   integer path (1 and 2 tokens), short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs
+//     fit beside this one's and have their rings full of weights when this kernel completes.
+//   floating-point path up to 8 tokens, and long integer-path ranges: the whole SM, 12 consumer warps (8 on the
+//     integer path) and a ring deep enough to keep HBM busy while 12 tiles are being consumed.  A consumer warp
+//     of the floating-point path is bound by instruction issue (about 20 issue cycles per packed word of 8
+//     weights, measured on registers alone), and since a GEMV may not read its activations before the kernel ahead
+//     of it has completed, only one kernel's consumers work on an SM at a time: three warps per scheduler beat two
+//     warps plus a waiting neighbour (decode step of the benchmark: 133 against 140 us).
+//   9..16 tokens: twice the MMA and activation work per tile and the whole SM, but 8 consumer warps: every tile a
+//     warp is working on is a tile that is not in flight (measured on the four layer shapes with the ring holding
+//     weights only: 8 warps 7.9 / 4.1 / 14.5 / 15.4 us, 10 warps 8.4 / 4.1 / 15.2 / 16.1 us; 12 warps do not fit the
+//     register file).
 __host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 8; }
 __host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
 // Shared memory a half-SM CTA asks for when two of its kind must not share an SM: with 228 KB per SM and 1 KB reserved
 // per CTA, two of these do not fit (2 x 115 KB), one beside a plain half-SM CTA (at most 110 KB) does.
 constexpr int kGemvSoloSmemBytes = 114 * 1024;
-// Packed bytes per CTA from which up to 8 tokens use the whole-SM configuration.  Measured with the same call back
-// to back, the whole SM wins from about 400 KB (4096 x 28672: 18.1 against 19.4 us); between calls of other sizes
-// the half-SM form overlaps with its neighbours and wins up to more (a decoder layer whose joined gate + up
-// projection has 412 KB per CTA: 41.2 against 46.8 us per layer).  At 472 KB (4096 x 32768) the whole SM is ahead
-// by 2 us either way.  The integer path has 8 consumer warps in both forms and crosses over later (562 KB per
-// CTA: 16.6 us half, 17.7 whole; 787 KB: 23.1 / 22.7; 899 KB: 30.7 / 26.0).
-constexpr int kGemvFullFromBytes = 440 * 1024;
+// Packed bytes per CTA from which the integer path uses the whole-SM configuration (8 consumer warps in both forms;
+// measured on int8 weights: 562 KB per CTA 16.6 us half, 17.7 whole; 787 KB: 23.1 / 22.7; 899 KB: 30.7 / 26.0).
 constexpr int kGemvFullFromBytesI8 = 704 * 1024;
 constexpr int kGemvMaxDevices = 64;            // devices the per-device caches cover
 constexpr int kGemvMaxStages = 48;
@@ -34,7 +36,7 @@ constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
 constexpr int kGemvStageBytes = 17408;        // 17 x 1024 >= 4 x 4256 and >= 2 x 8320
 constexpr int kGemvMaxM = 16;
-constexpr int kGemvI8MaxM = 2;                // int8 weights, up to this many tokens: the GEMV runs on the integer warp MMA
+constexpr int kGemvI8MaxM = 2;                // up to this many tokens the GEMV runs on the integer warp MMA (4-bit and int8 weights)
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
 // Workspace layout, shared with the GEMM so that one workspace serves every call of a stream:
 //   [0,16) status word | [256, 256+4*512) GEMV per-strip arrival counters | [4096, 20480) GEMM per-tile arrival
@@ -52,7 +54,7 @@ struct GemvPlan {
     int consumers;     // consumer warps
     int stages;        // ring depth
     bool full;         // whole-SM configuration
-    bool i8;           // integer path: int8 codes x activation pieces (W8, 1 or 2 tokens)
+    bool i8;           // integer path: codes x activation pieces on the integer warp MMA (1 or 2 tokens)
     int cluster;       // CTAs per cluster (1 = global mode: cut strips go through the workspace)
     int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster); global mode: CTAs that get tiles
     int xslot_bytes;   // cluster mode: bytes of one partial-sum slot in shared memory
