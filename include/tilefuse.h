@@ -22,6 +22,12 @@
  *   - Same inputs give bit-identical outputs (no atomics on results).
  *   - There is no CPU or other-GPU fallback: a device that is not compute capability
  *     10.x gives TF_ERR_ARCH.
+ *   - Thread safety: every entry point may be called from several host threads at once.  The
+ *     library's only state is per-device caches of immutable facts (device attributes, "this
+ *     kernel's attributes are set", occupancy answers) and the per-stream note above, all held
+ *     in atomics; a race on first use repeats an idempotent query.  The caller keeps calls that
+ *     share a workspace (or the fixed scratch of tf_gemv_w4a16_static) from overlapping on the
+ *     GPU, and makes the CUDA device current on the calling thread.
  */
 #ifndef TILEFUSE_H
 #define TILEFUSE_H
@@ -245,15 +251,19 @@ tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  *   32768) on devices with any SM count (at most 160 persistent CTAs are used); shapes beyond those limits
  *   are rejected with TF_ERR_SHAPE.
  *   The call never calls cudaMalloc, cudaFree or an allocating library routine.  The first call on a device
- *   looks up the array's device address (one-time set-up, done with that device current): make that first
- *   call before any stream capture.  Each call first clears, on `cuda_stream`, the part of the array that
- *   must start at zero.  All calls share the array: calls that overlap on the GPU (different streams) race
- *   on it, so serialise them.  The device status word is not readable through this call.
- *   Arguments, arithmetic and results are those of tf_gemv_w4a16.
+ *   (of either function below) looks up the array's device address and does every other one-time step a
+ *   launch of any shape can need (function attributes of all kernel variants, occupancy queries), with that
+ *   device current: make that first call before any stream capture.  Each call first clears, on
+ *   `cuda_stream`, the part of the array that must start at zero.  All calls share the array: calls that
+ *   overlap on the GPU (different streams) race on it, so serialise them.
+ *   Arguments, arithmetic and results are those of tf_gemv_w4a16.  What tf_device_status reports for a
+ *   workspace (a blob that does not match the arguments, a device-side wait that gave up) is reported for the
+ *   last static call of the current device by tf_gemv_w4a16_static_status, which synchronises `cuda_stream`.
  * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_ALIGN, TF_ERR_ARCH, TF_ERR_CUDA.
  */
 tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_bf16,
                                int M, int K, int N, void* cuda_stream);
+tf_status tf_gemv_w4a16_static_status(void* cuda_stream);
 
 /*
  * Second ablation arm (Section 5.5 separates the gain of fusing from the gain of the offline re-tiling of
@@ -290,6 +300,22 @@ size_t tf_gemv_awq_raw_workspace_size(int M, int K, int N, int group_size);
  * Pure host code apart from the device query; launches nothing.  Errors: TF_ERR_NULL, TF_ERR_SHAPE.
  */
 tf_status tf_gemv_plan(int bits, int M, int K, int N, int sm_count, int* out);
+
+/*
+ * Test hook for the failure path (the paper has no counterpart: its kernels run under a host runtime that owns
+ * error handling).  Every device-side wait of the GEMV and GEMM kernels is bounded; when one runs out, all
+ * roles of the CTA leave their loops, copies in flight are given time to land, tensor memory is freed, the
+ * kernel returns and the status word of the workspace becomes TF_ERR_TIMEOUT.  This call makes that happen on
+ * purpose, without faulting or hanging anything, for every tf_gemv_* / tf_gemm_* launch of this process that
+ * follows it:
+ *   wait_limit_kcycles   limit of a device-side wait in units of 1024 SM cycles (0 = the default, about 1 s);
+ *                        must be below 2^24.
+ *   drop_weight_copies   non-zero: the packed-weight producer issues no copies, so every wait for weights
+ *                        runs out after the limit (y is then left untouched).
+ * tf_debug_inject(0, 0) restores normal operation.  Process-wide, not for production use.
+ * Errors: TF_ERR_SHAPE (limit out of range).
+ */
+tf_status tf_debug_inject(unsigned wait_limit_kcycles, int drop_weight_copies);
 
 /* Scratch bytes the given operation needs for this shape (0 if none; 0 also if the shape
  * is illegal -- the compute call then reports TF_ERR_SHAPE). */

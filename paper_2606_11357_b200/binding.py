@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIG
 EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
-           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan")
+           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan", "tf_debug_inject", "tf_gemv_w4a16_static_status")
 
 
 class TileFuseError(RuntimeError):
@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.tf_gemv_w4a16_static.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_workspace_size.restype, L.tf_workspace_size.argtypes = c_size, [c_int] * 4
         L.tf_gemv_plan.restype, L.tf_gemv_plan.argtypes = c_int, [c_int] * 5 + [vp]
+        L.tf_debug_inject.restype, L.tf_debug_inject.argtypes = c_int, [ctypes.c_uint, c_int]
+        L.tf_gemv_w4a16_static_status.restype, L.tf_gemv_w4a16_static_status.argtypes = c_int, [vp]
         L.tf_dequant_bf16.restype, L.tf_dequant_bf16.argtypes = c_int, [vp, vp, c_int, c_int, c_int, vp]
         L.tf_gemv_awq_raw.restype = c_int
         L.tf_gemv_awq_raw.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, c_int, vp, c_size, vp]
@@ -193,6 +195,16 @@ def tf_gemv_w4a16_static(packed, a, y, M, K, N, stream=None) -> None:
     """tf_gemv_w4a16 for callers that cannot provide a workspace: scratch is a fixed array inside the library.
     Calls share that array, so do not let two of them overlap on the GPU."""
     _check("tf_gemv_w4a16_static", lib().tf_gemv_w4a16_static(_dev(packed), _dev(a), _dev(y), M, K, N, _stream(stream)))
+
+
+def tf_gemv_w4a16_static_status(stream=None) -> int:
+    return lib().tf_gemv_w4a16_static_status(_stream(stream))
+
+
+def tf_debug_inject(wait_limit_kcycles: int = 0, drop_weight_copies: bool = False) -> None:
+    """Failure-path test hook: shorten the device-side wait limit and/or make the weight producer issue nothing,
+    for every launch that follows; tf_debug_inject() restores normal operation."""
+    _check("tf_debug_inject", lib().tf_debug_inject(wait_limit_kcycles, 1 if drop_weight_copies else 0))
 
 
 def tf_gemv_w8a16(packed, a, y, M, K, N, workspace, stream=None) -> None:

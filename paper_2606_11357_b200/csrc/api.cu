@@ -2,6 +2,8 @@
 // other than a per-device cache of immutable device attributes.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "../../include/tilefuse.h"
 #include "kernels.h"
 #include "layout.h"
@@ -9,29 +11,34 @@
 namespace {
 
 struct DeviceInfo {
-    int known;      // 0 = not queried, 1 = ok (cc 10.x), -1 = wrong architecture, -2 = query failed
+    int known;      // 1 = ok (cc 10.x), -1 = wrong architecture
     int sm_count;
 };
-DeviceInfo g_devices[64];
+// Per device: 0 = not queried yet, else (sm_count << 2) | (2 = compute capability 10.x, 1 = another architecture).
+// One atomic word per device, so a host thread either sees nothing or a complete entry; two threads that query at the
+// same time store the same value.
+std::atomic<int> g_devices[64];
+std::atomic<uint32_t> g_debug_word{0};
 
 // Device attributes of the current device (cached after the first call on that device).
 tf_status device_info(DeviceInfo* out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
     if (dev < 0 || dev >= 64) return TF_ERR_CUDA;
-    DeviceInfo& d = g_devices[dev];
-    if (d.known == 0) {
+    int word = g_devices[dev].load(std::memory_order_acquire);
+    if (word == 0) {
         int major = 0, sms = 0;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
             cudaGetLastError();
             return TF_ERR_CUDA;
         }
-        d.sm_count = sms;
-        d.known = major == 10 ? 1 : -1;
+        word = (sms << 2) | (major == 10 ? 2 : 1);
+        g_devices[dev].store(word, std::memory_order_release);
     }
-    if (d.known != 1) return TF_ERR_ARCH;
-    *out = d;
+    if ((word & 3) != 2) return TF_ERR_ARCH;
+    out->known = 1;
+    out->sm_count = word >> 2;
     return TF_OK;
 }
 
@@ -79,6 +86,17 @@ tf_status gemm(int bits, const void* packed, const void* a, void* y, int M, int 
 }
 
 }  // namespace
+
+namespace tf {
+uint32_t debug_word() { return g_debug_word.load(std::memory_order_relaxed); }
+void set_debug_word(uint32_t word) { g_debug_word.store(word, std::memory_order_relaxed); }
+}  // namespace tf
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_debug_inject(unsigned wait_limit_kcycles, int drop_weight_copies) {
+    if (wait_limit_kcycles >= (1u << 24)) return TF_ERR_SHAPE;
+    tf::set_debug_word((wait_limit_kcycles << 8) | (drop_weight_copies ? 1u : 0u));
+    return TF_OK;
+}
 
 extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_w4a16(const void* packed, const void* a, void* y, int M, int K, int N,
                                    void* workspace, size_t workspace_bytes, void* stream) {

@@ -35,9 +35,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Gives up after about a second of polling, or as soon as another thread of the CTA
-// has given up (`*abort_flag` != 0).  On giving up it records `site` in the flag and returns false;
+// has given up (`abort_flag[0]` != 0).  On giving up it records `site` in the flag and returns false;
 // the caller must then leave its role loop and go to the common teardown.
+// `abort_flag` points at two words of shared memory: [0] the flag, [1] the limit of a wait in units of 1024
+// cycles, written once by the CTA's first thread from the kernel's `debug` argument (see wait_limit_kcycles).
 constexpr long long kWaitLimitCycles = 2000000000ll;
+// Kernel argument `debug` (0 in normal operation; set through tf_debug_inject for tests of the failure path):
+// bit 0 = the packed-weight producer issues no copies, so every wait for weights runs out; bits 8..31 = limit of a
+// wait in units of 1024 cycles (0 = the default of about a second).
+constexpr uint32_t kDebugDropWeights = 1u;
+__device__ __forceinline__ uint32_t wait_limit_kcycles(uint32_t debug) {
+    return (debug >> 8) != 0 ? (debug >> 8) : (uint32_t)(kWaitLimitCycles >> 10);
+}
+__device__ __forceinline__ bool wait_expired(long long t_begin, volatile uint32_t* abort_flag) {
+    return clock64() - t_begin > ((long long)abort_flag[1] << 10);
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint32_t site) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -46,7 +58,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 0xFFu) == 0) {
             if (*abort_flag != 0) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (wait_expired(t0, abort_flag)) {
                 *abort_flag = site;
                 return false;
             }

@@ -29,6 +29,9 @@
 // Every mbarrier wait is bounded; on a timeout all roles leave, TMEM is freed, the status word is set.
 #include <cuda.h>
 
+#include <atomic>
+#include <cstddef>
+
 #include "async.cuh"
 #include "common.cuh"
 #include "kernels.h"
@@ -117,10 +120,13 @@ struct GemmBarriers {
     uint64_t acc_full;
     uint64_t acc_empty;
     uint32_t tmem_base;
-    uint32_t abort_flag;
+    uint32_t abort_flag;        // [0] which wait gave up (0 = none) ...
+    uint32_t wait_kcycles;      // ... [1] limit of a wait in units of 1024 cycles (read by mbar_wait through the flag's address)
     uint32_t last_flag;
     uint32_t deferred_tile;     // 1 + the cut tile this CTA finishes with all its warps after the role loops (0 = none)
 };
+
+static_assert(offsetof(GemmBarriers, wait_kcycles) == offsetof(GemmBarriers, abort_flag) + 4, "mbar_wait reads the limit behind the flag");
 
 // One warp's share of the drain of a whole 128 x BT accumulator: the 8-token chunks `part`, `part + 3`, ... of its
 // lane quarter.  TMEM -> bf16 -> transposed through a 512-byte buffer -> one 16-byte store per lane (8 weight
@@ -176,7 +182,7 @@ template <int BITS, int BT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
             __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int n_tiles, int m_tiles, int aligned,
-            uint8_t* __restrict__ workspace) {
+            uint8_t* __restrict__ workspace, uint32_t debug) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kActStage = act_stage_bytes(BT);
@@ -220,6 +226,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
         mbar_init(smem_u32(&bars->acc_full), 1);
         mbar_init(smem_u32(&bars->acc_empty), 12);           // four epilogue warps + eight dequant warps (drain duty)
         bars->abort_flag = 0;
+        bars->wait_kcycles = wait_limit_kcycles(debug);
         bars->deferred_tile = 0;
         mbar_init_fence();
     }
@@ -273,6 +280,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     const int ws = wit % kWpStages;
                     ok = mbar_wait(smem_u32(&bars->wp_empty[ws]), ((wit / kWpStages) & 1) ^ 1, abort_flag, 0x300 + ws);
                     if (!ok) break;
+                    if (debug & kDebugDropWeights) continue;      // failure-path test: nothing ever arrives on wp_full
                     mbar_arrive_expect_tx(smem_u32(&bars->wp_full[ws]), nstrips * kTileBytes);
                     for (int q = 0; q < nstrips; ++q)
                         bulk_copy_g2s(smem_u32(wp_ring + ws * kWpStageBytes + q * kWpStripBytes),
@@ -627,17 +635,16 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
 
     // function attributes belong to one device: set them once per device and kernel (twice is harmless)
     constexpr int kMaxDevices = 64;
-    static bool configured_on[kMaxDevices] = {};
+    // (an atomic flag: two host threads may both find it unset and both set the attribute, which is harmless)
+    static std::atomic<bool> configured_on[kMaxDevices];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
-    bool unseen = dev < 0 || dev >= kMaxDevices;
-    bool& configured = unseen ? unseen : configured_on[dev];
-    if (unseen) configured = false;
-    if (!configured) {
+    const bool seen = dev >= 0 && dev < kMaxDevices;
+    if (!seen || !configured_on[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BITS, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              gemm_smem_bytes(BITS, BT));
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (seen) configured_on[dev].store(true, std::memory_order_release);
     }
     const int n_tiles = (N + kBN - 1) / kBN, m_tiles = (M + BT - 1) / BT;
     const long long units = (long long)n_tiles * m_tiles * (K / kTileK);
@@ -666,7 +673,7 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     cfg.numAttrs = 1;
     note_whole_sm_launch(stream);
     return cudaLaunchKernelEx(&cfg, gemm_kernel<BITS, BT>, map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K,
-                              N, ktiles, n_tiles, m_tiles, aligned, static_cast<uint8_t*>(workspace));
+                              N, ktiles, n_tiles, m_tiles, aligned, static_cast<uint8_t*>(workspace), debug_word());
 }
 
 template <int BITS>

@@ -133,7 +133,7 @@ template <int BITS, int MT, bool FULL, bool CL, bool I8>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
                    int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes,
-                   uint8_t* __restrict__ workspace) {
+                   uint8_t* __restrict__ workspace, uint32_t debug) {
     constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
@@ -192,7 +192,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         }
         mbar_init(seg_full0, nconsumers);               // every consumer warp has dropped its partial
         mbar_init(seg_free0, 1);                        // the reducer has read them
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = wait_limit_kcycles(debug);
         mbar_init_fence();
     }
     __syncthreads();
@@ -209,7 +210,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         // a strip boundary.  The loop is kept to a few dozen instructions per chunk: this warp shares its scheduler
         // with consumer warps that never idle.  It reads nothing but the packed weights, which are constants, so it
         // does not wait for the kernels before this one: the first ring fill is on its way while they finish.
-        if (lane == 0 && header_ok) {
+        if (lane == 0 && header_ok && (debug & kDebugDropWeights) == 0) {
             ChunkWalk walk(t0, ntiles, ktiles, blob + kHeaderBytes, kTileBytes);
             // first ring fill, weights only: they are constants, so they may be fetched before the dependency wait
             int cg = 0;
@@ -441,7 +442,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     const long long t_begin = clock64();
                     while (stage_tag[s] != (uint32_t)cg && !aborted) {
                         if (*abort_flag != 0) aborted = true;
-                        else if (clock64() - t_begin > kWaitLimitCycles) { *abort_flag = 0x280 + s; aborted = true; }
+                        else if (wait_expired(t_begin, abort_flag)) { *abort_flag = 0x280 + s; aborted = true; }
                     }
                     if (aborted) break;
                 }
@@ -752,12 +753,12 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 // How many clusters of `csize` CTAs the device can hold at once, for half-SM CTAs (two per SM) or whole-SM ones
 // (asked once per device).  0 if the question fails: cluster mode is then not used.
 static int max_resident_clusters(int csize, bool full) {
-    static int cached[kGemvMaxDevices][2][4];   // [device][full][log2 csize], 0 = not asked yet, -1 = failed
+    static std::atomic<int> cached[kGemvMaxDevices][2][4];   // [device][full][log2 csize], 0 = not asked yet, -1 = failed
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kGemvMaxDevices) return 0;
     const int slot = csize == 2 ? 1 : csize == 4 ? 2 : 3;
-    int& entry = cached[dev][full ? 1 : 0][slot];
-    if (entry == 0) {
+    int entry = cached[dev][full ? 1 : 0][slot].load(std::memory_order_relaxed);
+    if (entry == 0) {                           // two host threads may both ask: same answer, harmless
         int n = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(csize * 64, 1, 1);
@@ -780,6 +781,7 @@ static int max_resident_clusters(int csize, bool full) {
         }
         if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
         entry = n > 0 ? n : -1;
+        cached[dev][full ? 1 : 0][slot].store(entry, std::memory_order_relaxed);
     }
     return entry > 0 ? entry : 0;
 }
@@ -912,28 +914,54 @@ void note_launch(cudaStream_t stream, bool whole_sm) {
 void note_whole_sm_launch(cudaStream_t stream) { note_launch(stream, true); }
 
 
+// Function attributes belong to one device: set once per device and kernel instantiation.  The flag is atomic: two
+// host threads may both find it unset and both set the attributes, which is harmless.
+template <int BITS, int MT, bool FULL, bool CL, bool I8>
+static cudaError_t configure_one() {
+    static std::atomic<bool> configured_on[kGemvMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    const bool seen = dev >= 0 && dev < kGemvMaxDevices;
+    if (seen && configured_on[dev].load(std::memory_order_acquire)) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         FULL ? gemv_smem_budget(MT, FULL) : kGemvSoloSmemBytes);
+    if (e != cudaSuccess) return e;
+    // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
+    // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
+    // consecutive GEMVs of different shapes could not share an SM.
+    e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    if (seen) configured_on[dev].store(true, std::memory_order_release);
+    return cudaSuccess;
+}
+
+template <int BITS>
+static cudaError_t configure_bits() {
+    cudaError_t e = cudaSuccess;
+    auto all = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+    all(configure_one<BITS, 1, false, false, false>()); all(configure_one<BITS, 1, true, false, false>());
+    all(configure_one<BITS, 1, false, false, true>());  all(configure_one<BITS, 1, true, false, true>());
+    all(configure_one<BITS, 2, true, false, false>());
+    all(configure_one<BITS, 1, false, true, false>());  all(configure_one<BITS, 1, true, true, false>());
+    all(configure_one<BITS, 2, true, true, false>());
+    return e;
+}
+
+// Every one-time step a later launch on the current device could need (function attributes of every instantiation,
+// the cluster-occupancy answers), for callers that must not meet them inside a stream capture.
+cudaError_t configure_gemv_kernels() {
+    cudaError_t e = configure_bits<4>();
+    if (e == cudaSuccess) e = configure_bits<8>();
+    for (int c = 2; c <= 8; c *= 2) { max_resident_clusters(c, false); max_resident_clusters(c, true); }
+    return e;
+}
+
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
-    // function attributes belong to one device: set them once per device and kernel (twice is harmless)
-    static bool configured_on[kGemvMaxDevices] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
-    bool unseen = dev < 0 || dev >= kGemvMaxDevices;
-    bool& configured = unseen ? unseen : configured_on[dev];
-    if (unseen) configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             FULL ? gemv_smem_budget(MT, FULL) : kGemvSoloSmemBytes);
-        if (e != cudaSuccess) return e;
-        // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
-        // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
-        // consecutive GEMVs of different shapes could not share an SM.
-        e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    cudaError_t ce = configure_one<BITS, MT, FULL, CL, I8>();
+    if (ce != cudaSuccess) return ce;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.grid, 1, 1);
     cfg.blockDim = dim3(p.threads, 1, 1);
@@ -963,7 +991,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     }
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8>, static_cast<const uint8_t*>(blob),
                               static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
-                              p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace));
+                              p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace), debug_word());
 }
 
 template <int BITS>

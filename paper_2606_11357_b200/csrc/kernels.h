@@ -67,6 +67,13 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count);
 cudaError_t launch_gemv(int bits, const GemvPlan& plan, const void* blob, const void* a, void* y,
                         int M, int K, int N, void* workspace, cudaStream_t stream);
 
+// Do every one-time, per-device step of the GEMV launcher now (function attributes, occupancy queries).
+cudaError_t configure_gemv_kernels();
+
+// The `debug` argument every GEMV / GEMM launch passes to its kernel (0 unless tf_debug_inject set it; see async.cuh).
+uint32_t debug_word();
+void set_debug_word(uint32_t word);
+
 // Tell the GEMV launcher that a whole-SM kernel of this library (the GEMM) was launched on `stream`.
 void note_whole_sm_launch(cudaStream_t stream);
 

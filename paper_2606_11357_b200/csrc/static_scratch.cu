@@ -13,6 +13,8 @@
 // on the GPU (different streams, or graphs run concurrently) would race on it -- serialise them.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "../../include/tilefuse.h"
 #include "kernels.h"
 #include "layout.h"
@@ -25,19 +27,24 @@ constexpr size_t kStaticScratchBytes = tf::kGemvPartialOffset + (size_t)kStaticM
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 struct PerDevice {
-    int state;          // 0 = not set up, 1 = ready, -1 = wrong architecture
+    std::atomic<int> state;   // 0 = not set up, 1 = ready, -1 = wrong architecture; published after the fields below
     int sm_count;
-    void* scratch;      // device address of g_static_scratch on this device
+    void* scratch;            // device address of g_static_scratch on this device
 };
 PerDevice g_dev[64];
 
 // In host code `g_static_scratch` is only a handle for the symbol, not a device address: the address the
-// kernel needs comes from cudaGetSymbolAddress, asked once per device while that device is current.
+// kernel needs comes from cudaGetSymbolAddress, asked once per device while that device is current.  The same
+// first call does every other one-time step a GEMV launch can need (function attributes of every kernel variant,
+// occupancy queries), so that later calls of any shape do nothing but launch.  Two host threads that make their
+// first call at the same time both do the set-up and store the same values; `state` is written last (release), so
+// a thread that sees 1 also sees the address.
 tf_status setup_current_device(PerDevice** out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return TF_ERR_CUDA; }
     PerDevice& d = g_dev[dev];
-    if (d.state == 0) {
+    int state = d.state.load(std::memory_order_acquire);
+    if (state == 0) {
         int major = 0, sms = 0;
         void* ptr = nullptr;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -46,18 +53,20 @@ tf_status setup_current_device(PerDevice** out) {
             return TF_ERR_CUDA;
         }
         if (major != 10) {
-            d.state = -1;
+            state = -1;
         } else {
             if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
                 cudaGetLastError();
                 return TF_ERR_CUDA;
             }
+            if (tf::configure_gemv_kernels() != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
             d.scratch = ptr;
             d.sm_count = sms;
-            d.state = 1;
+            state = 1;
         }
+        d.state.store(state, std::memory_order_release);
     }
-    if (d.state != 1) return TF_ERR_ARCH;
+    if (state != 1) return TF_ERR_ARCH;
     *out = &d;
     return TF_OK;
 }
@@ -86,4 +95,14 @@ tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_b
         return TF_ERR_CUDA;
     }
     return TF_OK;
+}
+
+// The status word of the last tf_gemv_w4a16_static call on this device (every such call clears it before it
+// launches): synchronises `cuda_stream` and reads the first word of the fixed scratch array.
+extern "C" __attribute__((visibility("default")))
+tf_status tf_gemv_w4a16_static_status(void* cuda_stream) {
+    PerDevice* dev = nullptr;
+    tf_status st = setup_current_device(&dev);
+    if (st != TF_OK) return st;
+    return tf_device_status(dev->scratch, cuda_stream);
 }

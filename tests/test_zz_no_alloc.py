@@ -89,3 +89,19 @@ def test_static_scratch_gemv_chain_consumes_previous_output():
     q2 = copy.copy(p2)
     q2.a_bf16 = results[1][0]
     gu.check_against_oracle(q2, results[1][1])
+
+
+def test_static_scratch_status_reports_a_blob_mismatch():
+    """A blob that does not match the arguments is detected on the device: y stays untouched and the status reader of
+    the static entry point says so (a workspace call reports the same through tf_device_status)."""
+    p = wl.make_w4(2, 1024, 512, seed=105)
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    a = gu.to_device_bf16(p.a_bf16)
+    y = torch.full((2, 256), -5.0, dtype=torch.bfloat16, device="cuda")
+    tf.tf_gemv_w4a16_static(blob, a, y, 2, 1024, 256)              # N does not match the blob's header
+    assert tf.tf_gemv_w4a16_static_status() == 4                   # TF_ERR_BLOB
+    assert bool((y == -5.0).all())
+    y2 = torch.empty((2, 512), dtype=torch.bfloat16, device="cuda")
+    tf.tf_gemv_w4a16_static(blob, a, y2, 2, 1024, 512)             # the next call clears the word
+    assert tf.tf_gemv_w4a16_static_status() == 0
+    gu.check_against_oracle(p, gu.bits_of(y2))
