@@ -8,9 +8,13 @@ weights of a call (432 MB in total) have been pushed out of the 126 MB L2 before
 
   value      algorithmic GB/s of the whole step, inputs resident in HBM, launches replayed from a
              CUDA graph, timed with CUDA events on the launching stream (max over ranks).
-  e2e        the same step through the C-ABI calls one by one with HOST activations: pinned
-             host -> device copy of A and device -> host copy of Y inside the timed region.
+  e2e        the same step through the C-ABI calls, issued one by one inside the timed loop, with
+             HOST activations: pinned host -> device copy of A and device -> host copy of Y inside
+             the timed region (`graph_replay_value`: the same with the calls replayed from a graph).
   gemm       the prefill GEMM (M=2048, K=4096, N=14336, 1 % outlier channels) in TFLOP/s.
+  configs    the other benchmark configurations (0: GEMV 1x4096x4096; 3: W8A16 GEMM 1024x4096x4096
+             and GEMV 1x4096x14336; 4: GEMM 512x32768x4096 and GEMV 1x4096x32768), each in us and
+             GB/s or TFLOP/s with its fraction of the measured peak.
   roofline   achieved / measured-peak for the GEMV step (HBM bound); gemm.roofline likewise (tensor).
   cpu_baseline  the fp64 CPU oracle timed on this machine's host cores on a bounded sample.
 
@@ -197,7 +201,8 @@ def time_oracle_sample(repeats: int = 3):
             orc.solve(p)
     dt = (time.perf_counter() - t0) / repeats
     return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": oracle_threads(), "kind": "oracle",
-            "sample": f"fp64 oracle, the whole step (four Llama-3-8B layer shapes at M = 1, 4, 16), {repeats} passes "
+            "sample": f"the oracle as it stands (numpy: vectorised fp64 unpack and dequantization, one library fp64 matmul per call, BLAS threads as "
+                      f"counted in `cores`), the whole step (four Llama-3-8B layer shapes at M = 1, 4, 16), {repeats} passes "
                       f"({dt:.2f} s per pass, {nbytes / 1e6:.1f} MB algorithmic per pass)"}, dt, nbytes
 
 
@@ -221,7 +226,7 @@ def run_reference(args):
         "config": {"workload": "cfg1 decode GEMV sweep: Llama-3-8B layer shapes at M = 1, 4, 16 (each step: the oracle on the whole step, once)",
                    "l2": "n/a (CPU)"},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle_threads(), "kind": "oracle",
-                         "sample": "the whole step (four layer shapes at M = 1, 4, 16) once per timed step"},
+                         "sample": "the oracle as it stands (numpy fp64, one library matmul per call): the whole step (four layer shapes at M = 1, 4, 16) once per timed step"},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -366,7 +371,7 @@ def run_gpu(args):
     ev_comp = [torch.cuda.Event() for _ in range(2)]        # the set's GEMVs are done
     ev_out = [torch.cuda.Event() for _ in range(2)]         # the set's results are on the host
 
-    def e2e_step(s, first):
+    def e2e_step(s, first, use_graph):
         with torch.cuda.stream(s_in):
             if not first:
                 s_in.wait_event(ev_comp[s])                 # the step that last read these activations
@@ -376,24 +381,30 @@ def run_gpu(args):
             stream.wait_event(ev_in[s])
             if not first:
                 stream.wait_event(ev_out[s])                # the results of that step have left the device
-            step_graph[s].replay()
+            if use_graph:
+                step_graph[s].replay()
+            else:
+                enqueue_step(s)                             # twelve tf_gemv_w4a16 calls through the C ABI, one by one
             ev_comp[s].record(stream)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_comp[s])
             y_host_all[s].copy_(y_dev_all[s], non_blocking=True)
             ev_out[s].record(s_out)
 
-    e2e_step(0, True)
-    e2e_step(1, True)
-    torch.cuda.synchronize()
-    barrier()
-    t0 = time.perf_counter()
-    for i in range(e2e_steps):
-        e2e_step(i & 1, False)
-    torch.cuda.synchronize()
-    dt = time.perf_counter() - t0
-    dt = max_over_ranks(dt, dev)
-    e2e_value = world * step_bytes * e2e_steps / dt / 1e9
+    def e2e_run(use_graph):
+        e2e_step(0, True, use_graph)
+        e2e_step(1, True, use_graph)
+        torch.cuda.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i & 1, False, use_graph)
+        torch.cuda.synchronize()
+        dt = max_over_ranks(time.perf_counter() - t0, dev)
+        return world * step_bytes * e2e_steps / dt / 1e9
+
+    e2e_value = e2e_run(False)                   # the calls a user makes, issued inside the timed loop
+    e2e_graph_value = e2e_run(True)              # the same step captured once per weight set and replayed
 
     # ---- per-shape breakdown (graph of 2 launches on alternating copies; context for the step number) ---
     per_shape = []
@@ -502,6 +513,76 @@ def run_gpu(args):
                 "roofline": {"bound": "tensor", "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                              "frac": tfl / peaks["bf16_tflops"], "peak_kind": f"{peak_kind} (burst, cuBLAS bf16)",
                              "traffic": traffic.get("gemm_w4_cfg2_dram_bytes_per_launch")}}
+
+    # ---- the other configurations: 0 (GEMV 1x4096x4096), 3 (W8A16 GEMM and GEMV), 4 (32K stress GEMM and GEMV) -----
+    configs = None
+    if rank == 0 and not args.skip_gemm:
+        def gemv_case(label, prob, bits):
+            """us per call over rotating weight copies (more than twice the L2 in rotation), replayed from a graph."""
+            M, K, N = prob.M, prob.K, prob.N
+            host = (tf.tf_pack_awq(prob.qweight, prob.scales_f16, prob.qzeros, K, N) if bits == 4
+                    else tf.tf_pack_w8(prob.w_i8, prob.scales_f16, K, N))
+            nbytes = gemv_algorithmic_bytes(bits, M, K, N)
+            first = torch.from_numpy(host).to(dev)
+            blobs = [first] + [first.clone() for _ in range(int(300e6 // nbytes) + 1)]
+            a = torch.from_numpy(prob.a_bf16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            fn = tf.tf_gemv_w4a16 if bits == 4 else tf.tf_gemv_w8a16
+            g = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream):
+                fn(blobs[0], a, y, M, K, N, ws, stream=stream)
+                stream.synchronize()
+                with torch.cuda.graph(g, stream=stream):
+                    for b in blobs:
+                        fn(b, a, y, M, K, N, ws, stream=stream)
+                g.replay()
+                stream.synchronize()
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0.record(stream)
+                for _ in range(5):
+                    g.replay()
+                s1.record(stream)
+                stream.synchronize()
+            us = s0.elapsed_time(s1) * 1e3 / (5 * len(blobs))
+            gbs = nbytes / us / 1e3
+            return {"config": label, "call": f"tf_gemv_w{bits}a16", "M": M, "K": K, "N": N, "us": round(us, 3),
+                    "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
+                    "frac_of_8TBps": round(gbs / 8000.0, 4), "l2": f"{len(blobs)} weight copies in rotation"}
+
+        def gemm_case(label, prob, bits):
+            M, K, N = prob.M, prob.K, prob.N
+            host = (tf.tf_pack_awq(prob.qweight, prob.scales_f16, prob.qzeros, K, N) if bits == 4
+                    else tf.tf_pack_w8(prob.w_i8, prob.scales_f16, K, N))
+            blob = torch.from_numpy(host).to(dev)
+            a = torch.from_numpy(prob.a_bf16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            op = tf.TF_OP_GEMM_W4A16 if bits == 4 else tf.TF_OP_GEMM_W8A16
+            gws = torch.zeros(tf.tf_workspace_size(op, M, K, N), dtype=torch.uint8, device=dev)
+            fn = tf.tf_gemm_w4a16 if bits == 4 else tf.tf_gemm_w8a16
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream):
+                for _ in range(5):
+                    fn(blob, a, y, M, K, N, gws, stream=stream)
+                stream.synchronize()
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0.record(stream)
+                for _ in range(20):
+                    fn(blob, a, y, M, K, N, gws, stream=stream)
+                s1.record(stream)
+                stream.synchronize()
+            if tf.tf_device_status(gws, stream=stream) != 0:
+                raise SystemExit("GEMM device status word reports an error")
+            us = s0.elapsed_time(s1) * 1e3 / 20
+            tfl = 2.0 * M * K * N / us / 1e6
+            return {"config": label, "call": f"tf_gemm_w{bits}a16", "M": M, "K": K, "N": N, "us": round(us, 2),
+                    "TFLOPs": round(tfl, 1), "frac_of_bf16_burst_peak": round(tfl / peaks["bf16_tflops"], 4),
+                    "frac_of_2250_nominal": round(tfl / 2250.0, 4)}
+
+        configs = [gemv_case("cfg0", wl.config0(), 4),
+                   gemm_case("cfg3", wl.config3_gemm(), 8), gemv_case("cfg3", wl.config3_gemv(), 8),
+                   gemm_case("cfg4", wl.config4_gemm(), 4), gemv_case("cfg4", wl.config4_gemv(), 4)]
+        assert tf.tf_device_status(ws) == 0
 
     # ---- library kernels on the same sizes, as context (not part of the path, not a target) ----------------
     ceilings = None
@@ -661,15 +742,18 @@ def run_gpu(args):
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps,
-                "how": "per step one pinned-host -> device copy of the 12 activation blocks, 12 tf_gemv_w4a16 calls (a captured graph), one "
-                       "device -> pinned-host copy of the 12 results; copies and GEMVs of neighbouring steps overlap on three "
-                       "streams (two buffer sets); wall clock over all steps"},
+                "how": "per step one pinned-host -> device copy of the 12 activation blocks, 12 tf_gemv_w4a16 calls issued one by "
+                       "one through the C ABI inside the timed loop (no graph), one device -> pinned-host copy of the 12 results; "
+                       "copies and GEMVs of neighbouring steps overlap on three streams (two buffer sets); wall clock over all steps",
+                "graph_replay_value": e2e_graph_value,
+                "graph_replay_how": "the same loop with the 12 calls of a step captured once per weight set and replayed"},
         "gpu_launches": launches_per_step * steps_timed,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"{peak_kind} (copy bandwidth)",
                      "traffic": traffic.get("gemv_w4_step_dram_bytes"),
                      "kernel": "gemv_stream_kernel (all 12 launches of the step)"},
         "cpu_baseline": cpu_baseline,
+        "configs": configs,
         "per_shape": per_shape,
         "decode_layer": decode_layer,
         "ablation": ablation,
@@ -723,10 +807,14 @@ def run_profile_case(args):
     kind, bits = args.profile_case.split("_")
     big = bits.endswith("big")
     bits = int(bits[1])
+    shape = tuple(int(v) for v in args.profile_shape.lower().split("x")) if args.profile_shape else None
     if kind == "gemv" and big:
         prob = wl.config4_gemv()
     elif kind == "gemv":
-        prob = (wl.config1(args.profile_m or 1, 4096, 14336) if bits == 4 else wl.config3_gemv())
+        K, N = shape or (4096, 14336)
+        prob = (wl.config1(args.profile_m or 1, K, N) if bits == 4 else wl.config3_gemv())
+    elif big:
+        prob = wl.config4_gemm()
     else:
         prob = (wl.config2(args.profile_m or 2048) if bits == 4 else wl.config3_gemm())
     M, K, N = prob.M, prob.K, prob.N
@@ -755,9 +843,10 @@ def main(argv=None):
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--skip-gemm", action="store_true", help="leave out the prefill GEMM section")
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline")
-    ap.add_argument("--profile-case", choices=["gemv_w4", "gemv_w4big", "gemv_w8", "gemm_w4", "gemm_w8"], default=None,
+    ap.add_argument("--profile-case", choices=["gemv_w4", "gemv_w4big", "gemv_w8", "gemm_w4", "gemm_w4big", "gemm_w8"], default=None,
                     help="run --steps launches of one kernel on one case and exit (for ncu captures)")
     ap.add_argument("--profile-m", type=int, default=0, help="token count for --profile-case")
+    ap.add_argument("--profile-shape", default="", help="KxN of a config-1 layer shape for --profile-case gemv_w4 (default 4096x14336)")
     ap.add_argument("--gemm-sweep", action="store_true", help="time the W4A16 GEMM for M = 256..4096 on two K/N-swapped shapes")
     args = ap.parse_args(argv)
     if args.gemm_sweep:
