@@ -65,7 +65,7 @@ typedef enum tf_op {
 #define TF_MAX_M_GEMM   4096
 #define TF_TILE_K       128     /* k-extent of one packed tile = the AWQ group size */
 #define TF_TILE_N       64      /* n-extent of one packed tile (a "strip" of columns) */
-#define TF_WORKSPACE_HEAD_BYTES 20480   /* start of a workspace that must be zero before its first use */
+#define TF_WORKSPACE_ZERO_BYTES 1069056 /* start of a workspace that must be zero before its first use (or zero all of it) */
 
 /*
  * The packed blob (output of tf_pack_awq / tf_pack_w8).
@@ -185,10 +185,12 @@ tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int
  *   a_bf16   device, bf16 [M][K] row-major, leading dimension K.
  *   y_bf16   device, bf16 [M][N] row-major, leading dimension N; fully overwritten.
  *   workspace, workspace_bytes   device scratch of at least tf_workspace_size(op, M, K, N)
- *            bytes.  Its first TF_WORKSPACE_HEAD_BYTES bytes must be zero before the first call that
- *            uses it; every call leaves them zero again unless it reports an error there.  Bytes [0,16)
- *            hold the device status word read by tf_device_status; the rest holds arrival counters and
- *            the fp32 partial sums of the few column strips that are split between two CTAs.  GEMV and
+ *            bytes.  Its first TF_WORKSPACE_ZERO_BYTES bytes must be zero before the first call that
+ *            uses it; every call leaves them zero again unless it reports an error there (after an error
+ *            status, clear them before the next call).  Bytes [0,16) hold the device status word read by
+ *            tf_device_status; the rest holds arrival counters and the fp32 partial sums of the few
+ *            column strips that are split between CTAs (a partial sum announces itself: its slot is all
+ *            +0.0 until the sums, with +0.0 written as -0.0, arrive; no fence, no counter).  GEMV and
  *            GEMM calls lay the workspace out compatibly: one workspace of the largest size needed may
  *            serve every call of a stream, in any order.  Use one workspace per stream: calls that run
  *            concurrently must not share one.
@@ -202,7 +204,7 @@ tf_status tf_dequant_bf16(const void* packed, void* w_bf16, int bits, int K, int
  * activation makes every output of its token NaN there (the floating-point paths give Inf or NaN,
  * as IEEE arithmetic does).
  * Each persistent CTA streams one contiguous range of packed tiles; a strip of 64 output
- * columns that is cut between CTAs is summed in CTA order by the last CTA to finish it.
+ * columns that is cut between CTAs is summed in a fixed order by the CTA that holds its first tile.
  * The blob must be at least tf_packed_size(bits, K, N, 128) bytes for the K, N passed here.
  * Errors: TF_ERR_NULL, TF_ERR_SHAPE (M outside 1..16, K % 128, N % 8, limits), TF_ERR_ALIGN,
  *         TF_ERR_WORKSPACE, TF_ERR_ARCH, TF_ERR_CUDA.  A blob/argument mismatch is detected on
@@ -227,7 +229,7 @@ tf_status tf_gemv_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  * output tile whose K range is cut between CTAs is summed in fp32 through the workspace, in CTA
  * order, by the last CTA to finish its part, so results do not depend on timing.
  * Workspace: tf_workspace_size() bytes (tens of MB: two fp32 tile slots per CTA).  Its first
- * TF_WORKSPACE_HEAD_BYTES bytes (status word and arrival counters) must be zero before the first
+ * TF_WORKSPACE_ZERO_BYTES bytes (status word, arrival counters, the GEMV's slots) must be zero before the first
  * call that uses it; every call leaves them zero again unless it reports an error there.  One
  * workspace per stream (it may be the one the GEMV calls of that stream use): calls that run
  * concurrently must not share one.
@@ -245,8 +247,8 @@ tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  * counterpart to this call; it exists for hosts of this library that cannot give it device memory: a
  * plug-in in a process whose memory pool another framework owns, a thread that must stay out of the
  * allocator, code inside a stream capture.)
- *   Scratch (arrival counters, fp32 partial sums of strips cut between two CTAs, status word) is a fixed
- *   array of about 1.27 MB inside the library's device image: every GPU that loads the library holds it
+ *   Scratch (status word, fp32 partial sums of strips cut between CTAs) is a fixed array of 675,840 bytes
+ *   inside the library's device image: every GPU that loads the library holds it
  *   until the process exits.  It covers every shape tf_gemv_w4a16 accepts (1 <= M <= 16, K and N up to
  *   32768) on devices with any SM count (at most 160 persistent CTAs are used); shapes beyond those limits
  *   are rejected with TF_ERR_SHAPE.
@@ -258,7 +260,8 @@ tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
  *   overlap on the GPU (different streams) race on it, so serialise them.
  *   Arguments, arithmetic and results are those of tf_gemv_w4a16.  What tf_device_status reports for a
  *   workspace (a blob that does not match the arguments, a device-side wait that gave up) is reported for the
- *   last static call of the current device by tf_gemv_w4a16_static_status, which synchronises `cuda_stream`.
+ *   last static call of the current device by tf_gemv_w4a16_static_status, which synchronises `cuda_stream`
+ *   (and, when it reports an error, clears the whole array so that the next call starts clean).
  * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_ALIGN, TF_ERR_ARCH, TF_ERR_CUDA.
  */
 tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_bf16,

@@ -71,12 +71,13 @@ __host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
            kWpStages * 2 * wp_strip_bytes(bits) + 4 * kEpiWarpBytes + 8 * kDrainWarpBytes + 512;
 }
 
-// workspace: [0,16) status | [kGemmCounterOffset, +4 * tiles) arrival counters | partial accumulators, two
-// slots of 128 x BT fp32 per CTA (head and tail of its range)
+// workspace: [0,16) status | [kGemmCounterOffset, +4 * tiles) arrival counters | (the GEMV's partial-sum slots, not
+// touched here) | partial accumulators, two slots of 128 x BT fp32 per CTA (head and tail of its range)
 constexpr int kGemmCounterOffset = 4096;       // behind the GEMV's counters: the two kernels may share a workspace
 constexpr int kGemmMaxTiles = 4096;            // (32768 / 128) n-tiles x (4096 / 256) token tiles
-constexpr int kGemmPartialOffset = kGemmCounterOffset + 4 * kGemmMaxTiles;
-static_assert(kGemmPartialOffset == kWorkspaceHeadBytes && kGemmCounterOffset >= kGemvCounterEnd, "workspace layout shared with the GEMV");
+constexpr size_t kGemmPartialOffset = kWorkspaceZeroBytes;      // behind the GEMV's partial-sum slots, which must stay zero
+static_assert(kGemmCounterOffset + 4 * kGemmMaxTiles == kWorkspaceHeadBytes && kGemmCounterOffset >= kGemvStatusBytes,
+              "workspace layout shared with the GEMV");
 constexpr int kGemmMaxGrid = 160;
 
 __device__ __forceinline__ int unit_start(int cta, int total, int grid) {

@@ -127,6 +127,59 @@ __device__ __forceinline__ void store_strip(__nv_bfloat16* y, const float4 (&tot
     }
 }
 
+// Hand-over of a cut strip without a fence or a counter.  The partial-sum slots of a workspace are all +0.0 bits
+// between calls.  A contributor stores its sums with every +0.0 replaced by -0.0 (the same number), so a word that is
+// not +0.0 has arrived, whatever the order in which the memory system delivers the words.  The finisher reads a slot
+// until all of its words have arrived, adds it, and puts +0.0 back for the next call.  It waits for stores that were
+// issued at about the time it starts to look (every wait is bounded), and the critical path of a cut strip is one
+// trip to the L2 instead of three (stores acknowledged -> arrival counter returned -> partial sums loaded).
+__device__ __forceinline__ float4 never_plus_zero(float4 v) {
+    const uint32_t x = __float_as_uint(v.x), y = __float_as_uint(v.y), z = __float_as_uint(v.z), w = __float_as_uint(v.w);
+    return make_float4(__uint_as_float(x == 0u ? 0x80000000u : x), __uint_as_float(y == 0u ? 0x80000000u : y),
+                       __uint_as_float(z == 0u ? 0x80000000u : z), __uint_as_float(w == 0u ? 0x80000000u : w));
+}
+// `slot` already points at this lane's first float4 of the partial of the first of `count` (<= kBatch) consecutive
+// CTAs; rows of tokens >= M are neither written nor read.  The loads of all `count` partials are issued together (one
+// trip to the L2 per turn), then the partials are added to `acc` in CTA order and their slots cleared.  Returns false
+// if the wait ran out.  Kept out of line so that the polling loop does not take part in the register allocation of the
+// streaming kernel around it.
+template <int kVec, int kBatch>
+__device__ __noinline__ bool gather_partials(float4* slot, int count, int M, float4 (&acc)[kVec], volatile uint32_t* abort_flag, uint32_t site) {
+    constexpr int kSlotVec = kGemvSlotBytes / 16;
+    float4 v[kBatch][kVec];
+    const long long t_begin = clock64();
+    for (;;) {
+        bool here = true;
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) {
+                v[b][e] = make_float4(-0.f, -0.f, -0.f, -0.f);
+                if (b < count && 2 * e < M)                       // a real load on every turn of the loop, from the L2
+                    asm volatile("ld.relaxed.gpu.global.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                 : "=f"(v[b][e].x), "=f"(v[b][e].y), "=f"(v[b][e].z), "=f"(v[b][e].w)
+                                 : "l"(slot + b * kSlotVec + 32 * e) : "memory");
+            }
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+            for (int e = 0; e < kVec; ++e)
+                here = here && __float_as_uint(v[b][e].x) != 0u && __float_as_uint(v[b][e].y) != 0u &&
+                       __float_as_uint(v[b][e].z) != 0u && __float_as_uint(v[b][e].w) != 0u;
+        if (__all_sync(0xFFFFFFFFu, here)) break;
+        if (*abort_flag != 0) return false;
+        if (wait_expired(t_begin, abort_flag)) { *abort_flag = site; return false; }
+    }
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) {
+            acc[e].x += v[b][e].x; acc[e].y += v[b][e].y; acc[e].z += v[b][e].z; acc[e].w += v[b][e].w;
+            if (b < count && 2 * e < M) __stcg(slot + b * kSlotVec + 32 * e, make_float4(0.f, 0.f, 0.f, 0.f));
+        }
+    return true;
+}
+
 }  // namespace
 
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
@@ -177,7 +230,6 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     int fin_strip = -1, fin_first = 0;          // cluster mode: the strip this CTA finishes after the cluster barrier
 
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
-    uint32_t* counters = reinterpret_cast<uint32_t*>(workspace + kGemvCounterOffset);
     float* partials = reinterpret_cast<float*>(workspace + kGemvPartialOffset);
 
     const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N);
@@ -242,32 +294,35 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         // Lane l owns output elements 4(l + 32e) .. +3 of the [token][64 n] tile (e < kVec), as float4.
         if (header_ok) {
             constexpr int kVec = kTok * kTileN / 128;  // float4 per lane
-            float4 pre[kVec];                          // the other contributor's partial of the tail cut, fetched early
-            bool prefetched = false;
             int sidx = 0, i = 0;
             bool ok = true;
-            grid_dependency_wait();                    // y, counters and partial sums belong to earlier kernels until now
+            grid_dependency_wait();                    // y and the partial sums belong to earlier kernels until now
             while (i < ntiles && ok) {
                 const int tile0 = t0 + i;
                 const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
                 const int seg_len = min(ntiles - i, ktiles - T0);
                 const bool whole = seg_len == ktiles;
-                const bool is_last_seg = i + seg_len == ntiles;
                 const int c_first = range_owner(strip * ktiles - cbase, ctiles, cn);
                 const int c_last = range_owner(strip * ktiles + ktiles - 1 - cbase, ctiles, cn);
-                const int ncontrib = c_last - c_first + 1;
+                // Global mode, cut strip: the CTA that holds the strip's first tile finishes it.  Its part of the strip
+                // is the tail of its range; for every other contributor the strip is the head of the range, done early.
+                const bool finisher = (!CL || csize == 1) && !whole && c_first == crank;
 
-                // look ahead for the tail cut: two contributors, this CTA first, the other one already published
-                if ((!CL || csize == 1) && is_last_seg && !whole && ncontrib == 2 && c_first == cta) {
-                    uint32_t seen;
-                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counters + strip) : "memory");
-                    if (seen == 1u) {
-                        const float4* other = reinterpret_cast<const float4*>(
-                            partials + ((size_t)(cta + 1) * 2 + 0) * (kGemvMaxM * kTileN));            // its head cut
+                // While the consumers still work on this segment, collect what the other contributors have dropped
+                // (in CTA order; a partial has arrived when none of its words is +0.0, see gather_partials).
+                float4 others[kVec];
 #pragma unroll
-                        for (int e = 0; e < kVec; ++e) pre[e] = __ldcg(other + lane + 32 * e);
-                        prefetched = true;
+                for (int e = 0; e < kVec; ++e) others[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (finisher) {
+                    // one partial per trip: with four at once the finisher of a strip shared by four CTAs would wait one
+                    // trip instead of three, but the gathering code then needs 64 registers more and the whole step was
+                    // slower (measured: 125.7 against 122.6 us), 2 MB shapes gained 0.3 us, 9 MB shapes lost 1 us
+                    constexpr int kBatch = 1;
+                    for (int c = c_first + 1; c <= c_last && ok; c += kBatch) {
+                        float4* slot = reinterpret_cast<float4*>(partials + (size_t)c * (kGemvMaxM * kTileN)) + lane;
+                        ok = gather_partials<kVec, kBatch>(slot, min(kBatch, c_last - c + 1), M, others, abort_flag, 0x440);
                     }
+                    if (!ok) break;
                 }
 
                 ok = mbar_wait(seg_full0, sidx & 1, abort_flag, 0x400);
@@ -287,18 +342,13 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 __syncwarp();
                 if (lane == 0) mbar_arrive(seg_free0);                  // consumers may reuse the buffer
 
-                const bool finish_here = whole || (prefetched && is_last_seg);
-                float4 tot[kVec];
-                bool store = finish_here;
-                if (finish_here) {
+                if (whole || finisher) {
+                    // fixed order: the other contributors in CTA order, then this CTA
 #pragma unroll
                     for (int e = 0; e < kVec; ++e) {
-                        tot[e] = sum[e];
-                        if (!whole) {                                    // CTA order: this CTA, then the next one
-                            tot[e].x = (0.f + sum[e].x) + pre[e].x; tot[e].y = (0.f + sum[e].y) + pre[e].y;
-                            tot[e].z = (0.f + sum[e].z) + pre[e].z; tot[e].w = (0.f + sum[e].w) + pre[e].w;
-                        }
+                        sum[e].x += others[e].x; sum[e].y += others[e].y; sum[e].z += others[e].z; sum[e].w += others[e].w;
                     }
+                    store_strip<kVec>(y, sum, strip, M, N, lane);
                 } else if (CL && csize > 1) {
                     // cluster mode: hand the partial to the CTA that holds the strip's last tile (maybe this one);
                     // it adds the slots up in rank order after the cluster barrier at the end of the kernel
@@ -310,49 +360,12 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                                          "f"(sum[e].x), "f"(sum[e].y), "f"(sum[e].z), "f"(sum[e].w) : "memory");
                     if (c_last == crank) { fin_strip = strip; fin_first = c_first; }
                 } else {
-                    // publish this CTA's partial; the last contributor to arrive adds them up in CTA order
-                    const int slot = (i == 0) ? 0 : 1;
-                    float4* mine = reinterpret_cast<float4*>(partials + ((size_t)cta * 2 + slot) * (kGemvMaxM * kTileN));
+                    // Drop this CTA's partial for the finisher and go on: no fence, no counter.  The data says by itself
+                    // that it has arrived: the slot is all +0.0 between calls and no word stored here is +0.0.
+                    float4* mine = reinterpret_cast<float4*>(partials + (size_t)crank * (kGemvMaxM * kTileN)) + lane;
 #pragma unroll
-                    for (int e = 0; e < kVec; ++e) __stcg(mine + lane + 32 * e, sum[e]);
-                    __syncwarp();
-                    uint32_t prev = 0;
-                    if (lane == 0)
-                        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(counters + strip) : "memory");
-                    prev = __shfl_sync(0xffffffffu, prev, 0);
-                    if (prev == (uint32_t)(ncontrib - 1)) {
-#pragma unroll
-                        for (int e = 0; e < kVec; ++e) tot[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        // The sum runs in CTA order, but the loads of several contributors are issued together: one
-                        // L2 round trip per batch instead of one per contributor.  Rows of tokens >= M are never read.
-                        constexpr int kBatch = MT == 1 ? 4 : 2;
-                        for (int c0 = 0; c0 < ncontrib; c0 += kBatch) {
-                            float4 v[kBatch][kVec];
-#pragma unroll
-                            for (int b = 0; b < kBatch; ++b) {
-                                const int c = c0 + b;
-                                const int cslot = range_start(c_first + c, total_tiles, cn) >= strip * ktiles ? 0 : 1;
-                                const float4* src = reinterpret_cast<const float4*>(
-                                    partials + ((size_t)(c_first + c) * 2 + cslot) * (kGemvMaxM * kTileN)) + lane;
-#pragma unroll
-                                for (int e = 0; e < kVec; ++e) {
-                                    v[b][e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                    if (c < ncontrib && 2 * e < M) v[b][e] = __ldcg(src + 32 * e);
-                                }
-                            }
-#pragma unroll
-                            for (int b = 0; b < kBatch; ++b)
-#pragma unroll
-                                for (int e = 0; e < kVec; ++e) {
-                                    tot[e].x += v[b][e].x; tot[e].y += v[b][e].y; tot[e].z += v[b][e].z; tot[e].w += v[b][e].w;
-                                }
-                        }
-                        store = true;
-                    }
-                }
-                if (store) {
-                    store_strip<kVec>(y, tot, strip, M, N, lane);
-                    if (!whole && (!CL || csize == 1) && lane == 0) counters[strip] = 0;          // every contributor has arrived: reset
+                    for (int e = 0; e < kVec; ++e)
+                        if (2 * e < M) __stcg(mine + 32 * e, never_plus_zero(sum[e]));
                 }
                 i += seg_len;
                 ++sidx;

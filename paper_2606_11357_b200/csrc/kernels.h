@@ -39,14 +39,17 @@ constexpr int kGemvMaxM = 16;
 constexpr int kGemvI8MaxM = 2;                // up to this many tokens the GEMV runs on the integer warp MMA (4-bit and int8 weights)
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
 // Workspace layout, shared with the GEMM so that one workspace serves every call of a stream:
-//   [0,16) status word | [256, 256+4*512) GEMV per-strip arrival counters | [4096, 20480) GEMM per-tile arrival
-//   counters | from 20480: partial sums (written before they are read, so either kernel may leave anything there).
-// Everything below kWorkspaceHeadBytes is zero between calls.
+//   [0,16) status word | [4096, 20480) GEMM per-tile arrival counters | from 20480: one GEMV partial-sum slot
+//   (16 tokens x 64 columns fp32) per persistent CTA | behind them the GEMM's partial tiles (written before they are
+//   read, so the GEMM may leave anything there).
+// Everything below kWorkspaceZeroBytes is zero between calls: the GEMV's hand-over of a cut strip relies on its slots
+// being all +0.0 bits (see gather_partials in gemv.cu), the GEMM on its counters.
 constexpr int kWorkspaceHeadBytes = 20480;
-constexpr int kGemvCounterOffset = 256;
-constexpr int kGemvCounterEnd = 4096;         // the GEMV touches no counter beyond this
+constexpr int kGemvStatusBytes = 256;         // what the GEMV itself needs cleared besides its slots
 constexpr int kGemvPartialOffset = kWorkspaceHeadBytes;
-constexpr size_t kGemvWorkspaceBytes = kGemvPartialOffset + (size_t)kGemvMaxGrid * 2 * kGemvMaxM * 64 * 4;
+constexpr int kGemvSlotBytes = kGemvMaxM * 64 * 4;
+constexpr size_t kWorkspaceZeroBytes = kGemvPartialOffset + (size_t)kGemvMaxGrid * kGemvSlotBytes;
+constexpr size_t kGemvWorkspaceBytes = kWorkspaceZeroBytes;
 
 struct GemvPlan {
     int grid;          // persistent CTAs

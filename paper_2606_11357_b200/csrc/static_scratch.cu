@@ -3,14 +3,16 @@
 // Some hosts of this library cannot hand it a workspace: a plug-in inside a serving process whose memory
 // pool is owned (and already fully reserved) by another framework, a real-time thread that must never enter
 // the allocator, or code between cudaStreamBeginCapture and EndCapture, where cudaMalloc is not allowed.
-// For them the scratch the GEMV needs (arrival counters + the fp32 partial sums of strips cut between two
-// CTAs + the status word) lives in a fixed array in this library's own device image.  The entry point calls
+// For them the scratch the GEMV needs (the status word + one fp32 partial-sum slot per persistent CTA for strips cut
+// between CTAs) lives in a fixed array in this library's own device image.  The entry point calls
 // no cudaMalloc / cudaFree and no library routine that allocates.
 //
 // The array exists once per GPU that loads the library and stays until the process exits
-// (kStaticScratchBytes, about 1.27 MB).  All calls share it and it keeps whatever the last call left: the
-// bytes that must start at zero are cleared on the stream before every launch, and two calls that overlap
-// on the GPU (different streams, or graphs run concurrently) would race on it -- serialise them.
+// (kStaticScratchBytes, 675,840 bytes).  All calls share it and it keeps whatever the last call left: the status
+// word is cleared on the stream before every launch, the partial-sum slots are zero when the library is loaded and
+// every kernel that completes normally puts the zeros back (tf_gemv_w4a16_static_status clears the whole array when it
+// reports an error), and two calls that overlap on the GPU (different streams, or graphs run concurrently) would race
+// on it -- serialise them.
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -22,7 +24,7 @@
 namespace {
 
 constexpr int kStaticMaxGrid = 160;                       // persistent CTAs the scratch has room for
-constexpr size_t kStaticScratchBytes = tf::kGemvPartialOffset + (size_t)kStaticMaxGrid * 2 * tf::kGemvMaxM * 64 * 4;
+constexpr size_t kStaticScratchBytes = tf::kGemvPartialOffset + (size_t)kStaticMaxGrid * tf::kGemvSlotBytes;
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
@@ -87,7 +89,7 @@ tf_status tf_gemv_w4a16_static(const void* packed, const void* a_bf16, void* y_b
     if (st != TF_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // status word and arrival counters must start at zero; the partial sums are always written before read
-    if (cudaMemsetAsync(dev->scratch, 0, tf::kGemvCounterEnd, stream) != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
+    if (cudaMemsetAsync(dev->scratch, 0, tf::kGemvStatusBytes, stream) != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
     const int ctas = dev->sm_count < kStaticMaxGrid ? dev->sm_count : kStaticMaxGrid;
     const tf::GemvPlan plan = tf::plan_gemv(4, M, K, N, ctas);
     if (tf::launch_gemv(4, plan, packed, a_bf16, y_bf16, M, K, N, dev->scratch, stream) != cudaSuccess) {
@@ -104,5 +106,14 @@ tf_status tf_gemv_w4a16_static_status(void* cuda_stream) {
     PerDevice* dev = nullptr;
     tf_status st = setup_current_device(&dev);
     if (st != TF_OK) return st;
-    return tf_device_status(dev->scratch, cuda_stream);
+    st = tf_device_status(dev->scratch, cuda_stream);
+    if (st != TF_OK) {
+        // a kernel that gave up may have left partial sums behind: the next call needs the slots zero again
+        cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+        if (cudaMemsetAsync(dev->scratch, 0, kStaticScratchBytes, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess) {
+            cudaGetLastError();
+            return TF_ERR_CUDA;
+        }
+    }
+    return st;
 }

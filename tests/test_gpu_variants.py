@@ -56,12 +56,12 @@ def test_illegal_group_sizes_are_rejected():
     assert tf.tf_packed_size(8, 1024, 64, 1024) > 0
 
 
-@pytest.mark.parametrize("kind,M,K,N,zero_bytes", [("gemv", 1, 4096, 1024, 20480), ("gemv", 16, 4096, 4096, 20480),
-                                                   ("gemv", 4, 1536, 328, 20480), ("gemm", 300, 2048, 1096, 20480),
-                                                   ("gemm", 512, 4096, 640, 20480)])
+@pytest.mark.parametrize("kind,M,K,N,zero_bytes", [("gemv", 1, 4096, 1024, 1069056), ("gemv", 16, 4096, 4096, 1069056),
+                                                   ("gemv", 4, 1536, 328, 1069056), ("gemv", 3, 14336, 4096, 1069056), ("gemm", 300, 2048, 1096, 1069056),
+                                                   ("gemm", 512, 4096, 640, 1069056)])
 def test_workspace_head_is_left_zero(kind, M, K, N, zero_bytes):
-    """The status word and the arrival counters must be zero again after a call, so the same workspace serves
-    the next call without being cleared."""
+    """The status word, the arrival counters and the GEMV's partial-sum slots must be zero again after a call, so the
+    same workspace serves the next call without being cleared."""
     p = wl.make_w4(M, K, N, seed=900 + M)
     blob = torch.from_numpy(gu.pack(p)).cuda()
     a = gu.to_device_bf16(p.a_bf16)
@@ -228,7 +228,7 @@ def test_gemv_and_gemm_share_one_workspace():
             else:
                 tf.tf_gemm_w4a16(bm, am, ym, Mm, K, N, ws)
         assert tf.tf_device_status(ws) == 0
-        assert int(ws[:20480].to(torch.int32).sum().item()) == 0
+        assert int(ws[:1069056].to(torch.int32).sum().item()) == 0
         gu.check_against_oracle(pv, gu.bits_of(yv))
         gu.check_against_oracle(pm, gu.bits_of(ym))
 
