@@ -180,6 +180,45 @@ __device__ __noinline__ bool gather_partials(float4* slot, int count, int M, flo
     return true;
 }
 
+// The same hand-over taken row pair by row pair: for float4 index e (token rows 2e, 2e + 1) the words of up to four
+// consecutive CTAs' partials are requested together, so a strip shared by many CTAs and few tokens costs one trip per
+// row pair instead of one per contributor, in 16 registers.  `slot` as above; adds to acc[e] in CTA order.
+template <int kVec>
+__device__ __noinline__ bool gather_rows(float4* slot, int count, int M, float4 (&acc)[kVec], volatile uint32_t* abort_flag, uint32_t site) {
+    constexpr int kSlotVec = kGemvSlotBytes / 16;
+    const long long t_begin = clock64();
+    for (int e = 0; e < kVec && 2 * e < M; ++e) {
+        float4 v[4];
+        for (;;) {
+            bool here = true;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                v[b] = make_float4(-0.f, -0.f, -0.f, -0.f);
+                if (b < count)
+                    asm volatile("ld.relaxed.gpu.global.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                 : "=f"(v[b].x), "=f"(v[b].y), "=f"(v[b].z), "=f"(v[b].w) : "l"(slot + b * kSlotVec + 32 * e) : "memory");
+            }
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                here = here && __float_as_uint(v[b].x) != 0u && __float_as_uint(v[b].y) != 0u && __float_as_uint(v[b].z) != 0u &&
+                       __float_as_uint(v[b].w) != 0u;
+            if (__all_sync(0xFFFFFFFFu, here)) break;
+            if (*abort_flag != 0) return false;
+            if (wait_expired(t_begin, abort_flag)) { *abort_flag = site; return false; }
+        }
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            a.x += v[b].x; a.y += v[b].y; a.z += v[b].z; a.w += v[b].w;
+            if (b < count) __stcg(slot + b * kSlotVec + 32 * e, make_float4(0.f, 0.f, 0.f, 0.f));
+        }
+#pragma unroll
+        for (int k = 0; k < kVec; ++k)
+            if (k == e) { acc[k].x += a.x; acc[k].y += a.y; acc[k].z += a.z; acc[k].w += a.w; }
+    }
+    return true;
+}
+
 }  // namespace
 
 template <int BITS, int MT, bool FULL, bool CL, bool I8>
@@ -318,9 +357,16 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     // trip instead of three, but the gathering code then needs 64 registers more and the whole step was
                     // slower (measured: 125.7 against 122.6 us), 2 MB shapes gained 0.3 us, 9 MB shapes lost 1 us
                     constexpr int kBatch = 1;
-                    for (int c = c_first + 1; c <= c_last && ok; c += kBatch) {
-                        float4* slot = reinterpret_cast<float4*>(partials + (size_t)c * (kGemvMaxM * kTileN)) + lane;
-                        ok = gather_partials<kVec, kBatch>(slot, min(kBatch, c_last - c + 1), M, others, abort_flag, 0x440);
+                    const int nothers = c_last - c_first;
+                    if (nothers > 1 && nothers <= 4 && (M + 1) / 2 < nothers) {
+                        // more contributors than pairs of token rows: row pair by row pair, all contributors at once
+                        float4* slot = reinterpret_cast<float4*>(partials + (size_t)(c_first + 1) * (kGemvMaxM * kTileN)) + lane;
+                        ok = gather_rows<kVec>(slot, nothers, M, others, abort_flag, 0x450);
+                    } else {
+                        for (int c = c_first + 1; c <= c_last && ok; c += kBatch) {
+                            float4* slot = reinterpret_cast<float4*>(partials + (size_t)c * (kGemvMaxM * kTileN)) + lane;
+                            ok = gather_partials<kVec, kBatch>(slot, min(kBatch, c_last - c + 1), M, others, abort_flag, 0x440);
+                        }
                     }
                     if (!ok) break;
                 }
