@@ -78,6 +78,7 @@ typedef enum tf_op {
  *
  *   blob   = header (256 bytes) | tile(strip 0, ktile 0) | tile(0,1) | ... | tile(1,0) | ...
  *   W4 tile (4256 bytes) = 4096 B weights | 64 fp16 scales (128 B) | 64 4-bit zeros (32 B)
+ *           (group size 64 / 32: two / four scale blocks, then as many zero blocks: 4416 / 4736 bytes)
  *   W8 tile (8320 bytes) = 8192 B weights | 64 fp16 scales (128 B)
  *
  * Inside a tile the weights are stored in the register order of the tensor-core operand
@@ -92,19 +93,20 @@ typedef struct tf_blob_header {
     uint32_t bits;         /* 4 or 8 */
     uint32_t K;
     uint32_t N;
-    uint32_t group_size;   /* as given to the packer; a multiple of TF_TILE_K */
+    uint32_t group_size;   /* as given to the packer; a multiple of TF_TILE_K, or 64 / 32 (4-bit) */
     uint32_t n_padded;     /* N rounded up to a multiple of TF_TILE_N */
     uint32_t strips;       /* n_padded / TF_TILE_N */
     uint32_t ktiles;       /* K / TF_TILE_K */
-    uint32_t tile_bytes;   /* 4256 (W4) or 8320 (W8) */
+    uint32_t tile_bytes;   /* 4256 (W4; 4416 / 4736 for group size 64 / 32) or 8320 (W8) */
     uint64_t tiles_offset; /* 256 */
     uint64_t total_bytes;  /* = tf_packed_size(bits, K, N, group_size) */
     uint8_t  reserved[200];
 } tf_blob_header;
 
 /* Bytes of the packed blob, or 0 if the shape is illegal.
- * Legal: bits in {4, 8}; 128 <= K <= TF_MAX_DIM; 8 <= N <= TF_MAX_DIM; N % 8 == 0;
- * group_size % 128 == 0; K % group_size == 0. */
+ * Legal: bits in {4, 8}; 128 <= K <= TF_MAX_DIM; 8 <= N <= TF_MAX_DIM; N % 8 == 0; K % group_size == 0;
+ * group_size % 128 == 0, or, for bits == 4, group_size 64 or 32 (the tile then carries two or four
+ * scale and zero-point blocks, group after group along k: 4416 or 4736 bytes per tile). */
 size_t tf_packed_size(int bits, int K, int N, int group_size);
 
 /*
@@ -241,6 +243,24 @@ tf_status tf_gemm_w4a16(const void* packed, const void* a_bf16, void* y_bf16,
 tf_status tf_gemm_w8a16(const void* packed, const void* a_bf16, void* y_bf16,
                         int M, int K, int N, void* workspace, size_t workspace_bytes,
                         void* cuda_stream);
+
+/*
+ * The same two W4A16 operations for blobs packed with any legal group size (Section 2.2: group-wise
+ * quantization; 128 is the paper's and the default, 64 and 32 are the other sizes in common use).  group_size
+ * must be the one given to tf_pack_awq; tf_gemv_w4a16 / tf_gemm_w4a16 are these calls with group_size = 128
+ * and serve every blob whose group size is a multiple of 128.  With two or four groups per tile the GEMV
+ * takes its floating-point path for every token count (scale applied to the fp32 sum of each group), the
+ * GEMM reads the scale and zero point of each 64- or 32-deep slice of its dequantization job; everything
+ * else, including workspace size and layout, is unchanged.
+ * Errors: as tf_gemv_w4a16 / tf_gemm_w4a16; TF_ERR_SHAPE also for an illegal group size; a blob packed with
+ * another group size is detected on the device (TF_ERR_BLOB, y untouched).
+ */
+tf_status tf_gemv_w4a16_grouped(const void* packed, const void* a_bf16, void* y_bf16,
+                                int M, int K, int N, int group_size, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream);
+tf_status tf_gemm_w4a16_grouped(const void* packed, const void* a_bf16, void* y_bf16,
+                                int M, int K, int N, int group_size, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream);
 
 /*
  * tf_gemv_w4a16 without a caller-provided workspace and without any allocation.  (The paper has no

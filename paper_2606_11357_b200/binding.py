@@ -23,7 +23,8 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_NULL", 2: "TF_ERR_SHAPE", 3: "TF_ERR_ALIG
 EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_unpack_w4", "tf_unpack_w8",
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
-           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan", "tf_debug_inject", "tf_gemv_w4a16_static_status")
+           "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan", "tf_debug_inject", "tf_gemv_w4a16_static_status",
+           "tf_gemv_w4a16_grouped", "tf_gemm_w4a16_grouped")
 
 
 class TileFuseError(RuntimeError):
@@ -52,6 +53,9 @@ def lib() -> ctypes.CDLL:
         for name in ("tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16"):
             fn = getattr(L, name)
             fn.restype, fn.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, vp, c_size, vp]
+        for name in ("tf_gemv_w4a16_grouped", "tf_gemm_w4a16_grouped"):
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, c_int, vp, c_size, vp]
         L.tf_gemv_w4a16_static.restype = c_int
         L.tf_gemv_w4a16_static.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_workspace_size.restype, L.tf_workspace_size.argtypes = c_size, [c_int] * 4
@@ -189,6 +193,21 @@ def _linear(name, packed, a, y, M, K, N, workspace, stream):
 def tf_gemv_w4a16(packed, a, y, M, K, N, workspace, stream=None) -> None:
     """a: bfloat16 [M,K], y: bfloat16 [M,N] CUDA tensors; asynchronous on the stream."""
     _linear("tf_gemv_w4a16", packed, a, y, M, K, N, workspace, stream)
+
+
+def _linear_grouped(name, packed, a, y, M, K, N, group_size, workspace, stream):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(name, getattr(lib(), name)(_dev(packed), _dev(a), _dev(y), M, K, N, group_size, _dev(workspace), ws_bytes,
+                                      _stream(stream)))
+
+
+def tf_gemv_w4a16_grouped(packed, a, y, M, K, N, group_size, workspace, stream=None) -> None:
+    """tf_gemv_w4a16 for a blob packed with `group_size` (32, 64 or a multiple of 128)."""
+    _linear_grouped("tf_gemv_w4a16_grouped", packed, a, y, M, K, N, group_size, workspace, stream)
+
+
+def tf_gemm_w4a16_grouped(packed, a, y, M, K, N, group_size, workspace, stream=None) -> None:
+    _linear_grouped("tf_gemm_w4a16_grouped", packed, a, y, M, K, N, group_size, workspace, stream)
 
 
 def tf_gemv_w4a16_static(packed, a, y, M, K, N, stream=None) -> None:

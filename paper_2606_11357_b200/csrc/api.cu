@@ -45,17 +45,17 @@ tf_status device_info(DeviceInfo* out) {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 tf_status check_linear_args(int bits, const void* packed, const void* a, void* y, int M, int K, int N,
-                            int max_m) {
+                            int max_m, int group_size) {
     if (!packed || !a || !y) return TF_ERR_NULL;
     if (M < 1 || M > max_m) return TF_ERR_SHAPE;
-    if (tf_packed_size(bits, K, N, tf::kTileK) == 0) return TF_ERR_SHAPE;
+    if (tf_packed_size(bits, K, N, group_size) == 0) return TF_ERR_SHAPE;
     if (!aligned16(packed) || !aligned16(a) || !aligned16(y)) return TF_ERR_ALIGN;
     return TF_OK;
 }
 
 tf_status gemv(int bits, const void* packed, const void* a, void* y, int M, int K, int N, void* workspace,
-               size_t workspace_bytes, void* stream) {
-    tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMV);
+               size_t workspace_bytes, void* stream, int group_size = tf::kTileK) {
+    tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMV, group_size);
     if (st != TF_OK) return st;
     if (workspace == nullptr || workspace_bytes < tf::kGemvWorkspaceBytes) return TF_ERR_WORKSPACE;
     if (!aligned16(workspace)) return TF_ERR_ALIGN;
@@ -63,15 +63,15 @@ tf_status gemv(int bits, const void* packed, const void* a, void* y, int M, int 
     st = device_info(&dev);
     if (st != TF_OK) return st;
     if (dev.sm_count > tf::kGemvMaxGrid) dev.sm_count = tf::kGemvMaxGrid;
-    const tf::GemvPlan plan = tf::plan_gemv(bits, M, K, N, dev.sm_count);
+    const tf::GemvPlan plan = tf::plan_gemv(bits, M, K, N, dev.sm_count, tf::groups_per_tile(group_size));
     cudaError_t e = tf::launch_gemv(bits, plan, packed, a, y, M, K, N, workspace, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
     return TF_OK;
 }
 
 tf_status gemm(int bits, const void* packed, const void* a, void* y, int M, int K, int N, void* workspace,
-               size_t workspace_bytes, void* stream) {
-    tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMM);
+               size_t workspace_bytes, void* stream, int group_size = tf::kTileK) {
+    tf_status st = check_linear_args(bits, packed, a, y, M, K, N, TF_MAX_M_GEMM, group_size);
     if (st != TF_OK) return st;
     const size_t need = tf_workspace_size(bits == 4 ? TF_OP_GEMM_W4A16 : TF_OP_GEMM_W8A16, M, K, N);
     if (workspace == nullptr || workspace_bytes < need) return TF_ERR_WORKSPACE;
@@ -80,7 +80,7 @@ tf_status gemm(int bits, const void* packed, const void* a, void* y, int M, int 
     st = device_info(&dev);
     if (st != TF_OK) return st;
     cudaError_t e = tf::launch_gemm(bits, packed, a, y, M, K, N, workspace, workspace_bytes, dev.sm_count,
-                                    static_cast<cudaStream_t>(stream));
+                                    static_cast<cudaStream_t>(stream), tf::groups_per_tile(group_size));
     if (e != cudaSuccess) { cudaGetLastError(); return TF_ERR_CUDA; }
     return TF_OK;
 }
@@ -113,6 +113,15 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_w4a16(const 
 extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_w8a16(const void* packed, const void* a, void* y, int M, int K, int N,
                                    void* workspace, size_t workspace_bytes, void* stream) {
     return gemm(8, packed, a, y, M, K, N, workspace, workspace_bytes, stream);
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_w4a16_grouped(const void* packed, const void* a, void* y, int M, int K,
+                                   int N, int group_size, void* workspace, size_t workspace_bytes, void* stream) {
+    return gemv(4, packed, a, y, M, K, N, workspace, workspace_bytes, stream, group_size);
+}
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_w4a16_grouped(const void* packed, const void* a, void* y, int M, int K,
+                                   int N, int group_size, void* workspace, size_t workspace_bytes, void* stream) {
+    return gemm(4, packed, a, y, M, K, N, workspace, workspace_bytes, stream, group_size);
 }
 
 extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_plan(int bits, int M, int K, int N, int sm_count, int* out) {

@@ -88,6 +88,16 @@ __device__ __forceinline__ bool header_matches(const void* blob, uint32_t bits, 
     return h.x == kMagic && h.y == kBlobVersion && h.z == bits && h.w == K && h2.x == N;
 }
 
+// The group size recorded in the header, and whether it fits a kernel built for G groups per tile (G = 1: any
+// multiple of the tile's k-extent; G = 2, 4: exactly 128 / G).
+__device__ __forceinline__ uint32_t header_group_size(const void* blob) {
+    return __ldg(reinterpret_cast<const uint32_t*>(blob) + 5);
+}
+__device__ __forceinline__ bool group_size_fits(const void* blob, int G) {
+    const uint32_t gs = header_group_size(blob);
+    return G == 1 ? (gs >= (uint32_t)kTileK && gs % kTileK == 0) : gs == (uint32_t)(kTileK / G);
+}
+
 __device__ __forceinline__ float fp16_bits_to_float(uint16_t h) {
     return __half2float(__ushort_as_half(h));
 }

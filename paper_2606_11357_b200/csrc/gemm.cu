@@ -51,13 +51,16 @@ constexpr int kTmemCols = 512;
 constexpr int kMaxActStages = 12;
 constexpr int kWpStages = 3;              // packed-weight ring (one stage = the two strip tiles of one k-tile)
 
-__host__ __device__ constexpr int wp_strip_bytes(int bits) { return bits == 4 ? 4352 : 8320; }
+// one packed tile of the ring, rounded up to a multiple of 128 bytes (G = groups per tile: 4256, 4416 or 4736 bytes of tile)
+__host__ __device__ constexpr int wp_strip_bytes(int bits, int G = 1) { return bits == 4 ? (G == 1 ? 4352 : G == 2 ? 4480 : 4736) : 8320; }
 __host__ __device__ constexpr int act_stage_bytes(int bt) { return bt * kBK * 2; }
 // activation ring depth: as deep as fits beside the packed ring, at most kMaxActStages
-__host__ __device__ constexpr int act_stages(int bits, int bt) {
-    return (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt) > kMaxActStages
+constexpr int kGemmSmemMax = 227 * 1024;  // dynamic shared memory one CTA may ask for
+constexpr int kGemmSmemFixed = 1024 /*alignment slack*/ + 4 * 1024 /*epilogue warps*/ + 8 * 512 /*drain duty*/ + 512 /*barriers*/;
+__host__ __device__ constexpr int act_stages(int bits, int bt, int G = 1) {
+    return (kGemmSmemMax - kGemmSmemFixed - kWpStages * 2 * wp_strip_bytes(bits, G)) / act_stage_bytes(bt) > kMaxActStages
                ? kMaxActStages
-               : (220 * 1024 - kWpStages * 2 * wp_strip_bytes(bits)) / act_stage_bytes(bt);
+               : (kGemmSmemMax - kGemmSmemFixed - kWpStages * 2 * wp_strip_bytes(bits, G)) / act_stage_bytes(bt);
 }
 // A pipeline stage is 128 k: two 64-k activation sub-tiles and 64 operand columns, one barrier that fills (activations
 // landed + operand stored) and one that drains (MMAs done).  The thread that issues the MMAs pays a fixed price per
@@ -66,10 +69,13 @@ __host__ __device__ constexpr int act_stages(int bits, int bt) {
 // tile execute in about 520, and it -- not the tensor core -- set the pace.
 constexpr int kEpiWarpBytes = 1024;       // per epilogue warp: 16 tokens x 32 columns of bf16, for the transpose
 constexpr int kDrainWarpBytes = 512;      // per dequant warp: 8 tokens x 32 columns, for its share of an accumulator drain
-__host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt) {
-    return 1024 /*alignment slack*/ + act_stages(bits, bt) * act_stage_bytes(bt) +
-           kWpStages * 2 * wp_strip_bytes(bits) + 4 * kEpiWarpBytes + 8 * kDrainWarpBytes + 512;
+__host__ __device__ constexpr int gemm_smem_bytes(int bits, int bt, int G = 1) {
+    return 1024 /*alignment slack*/ + act_stages(bits, bt, G) * act_stage_bytes(bt) +
+           kWpStages * 2 * wp_strip_bytes(bits, G) + 4 * kEpiWarpBytes + 8 * kDrainWarpBytes + 512;
 }
+static_assert(kGemmSmemFixed == 1024 + 4 * kEpiWarpBytes + 8 * kDrainWarpBytes + 512, "act_stages budgets for exactly these");
+static_assert(gemm_smem_bytes(4, 256, 1) <= kGemmSmemMax && gemm_smem_bytes(4, 128, 2) <= kGemmSmemMax &&
+              gemm_smem_bytes(4, 128, 4) <= kGemmSmemMax && gemm_smem_bytes(8, 128, 1) <= kGemmSmemMax, "shared memory budget");
 
 // workspace: [0,16) status | [kGemmCounterOffset, +4 * tiles) arrival counters | (the GEMV's partial-sum slots, not
 // touched here) | partial accumulators, two slots of 128 x BT fp32 per CTA (head and tail of its range)
@@ -179,26 +185,28 @@ __device__ __forceinline__ uint32_t bf16_dup(float v) {
 
 }  // namespace
 
-template <int BITS, int BT>
+// G = groups per tile: 1 for group sizes that are multiples of 128, 2 / 4 for the 4-bit group sizes 64 / 32.
+template <int BITS, int BT, int G = 1>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restrict__ blob,
             __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int n_tiles, int m_tiles, int aligned,
             uint8_t* __restrict__ workspace, uint32_t debug) {
-    constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
+    static_assert(G == 1 || BITS == 4, "several groups per tile: the 4-bit format only");
+    constexpr int kTileBytes = tile_bytes(BITS, G);
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kActStage = act_stage_bytes(BT);
     constexpr int kSub = 2;                                           // 64-k sub-steps per pipeline stage
-    constexpr int kStages = act_stages(BITS, BT) / kSub < kMaxDepth ? act_stages(BITS, BT) / kSub : kMaxDepth;
+    constexpr int kStages = act_stages(BITS, BT, G) / kSub < kMaxDepth ? act_stages(BITS, BT, G) / kSub : kMaxDepth;
     constexpr int kUStage = kSub * kActStage;
     static_assert(kStages >= 2, "the pipeline needs two stages");
-    constexpr int kWpStripBytes = wp_strip_bytes(BITS);
+    constexpr int kWpStripBytes = wp_strip_bytes(BITS, G);
     constexpr int kWpStageBytes = 2 * kWpStripBytes;
     constexpr uint32_t kIdesc = umma_idesc_bf16(kBN, BT);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* act_ring = smem;                                        // kStages x kActStage   (1024-aligned)
-    uint8_t* wp_ring = act_ring + act_stages(BITS, BT) * kActStage;  // kWpStages x packed tiles
+    uint8_t* wp_ring = act_ring + act_stages(BITS, BT, G) * kActStage;  // kWpStages x packed tiles
     uint8_t* epi_buf = wp_ring + kWpStages * kWpStageBytes;          // 4 x kEpiWarpBytes
     uint8_t* drain_buf = epi_buf + 4 * kEpiWarpBytes;                // 8 x kDrainWarpBytes
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(drain_buf + 8 * kDrainWarpBytes);
@@ -212,7 +220,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     const int u_end = aligned ? unit_start(blockIdx.x + 1, total_tiles, gridDim.x) * ktiles : unit_start(blockIdx.x + 1, total_units, gridDim.x);
     const Segments segs(u_begin, u_end, ktiles);
     const int strips = (N + kTileN - 1) / kTileN;
-    const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N);
+    const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N) && group_size_fits(blob, G);
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
 
     if (threadIdx.x == 0) {
@@ -360,37 +368,48 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
                     if (!ok) break;
                     const uint8_t* tile_smem = wp_ring + ws * kWpStageBytes + strip_sel * kWpStripBytes;
                     uint32_t op[2][16];                        // [block][register of the 16x256b.x4 store]
-                    // scales of rows (w0,g), (w0,g+8), (w0+1,g), (w0+1,g+8)
-                    const uint2 sc = *(reinterpret_cast<const uint2*>(tile_smem + kWeightBytes + g * 16) + (q & 1));
-                    const uint32_t sw[2] = {sc.x, sc.y};
+                    // scales of rows (w0,g), (w0,g+8), (w0+1,g), (w0+1,g+8), split into two exact bf16 parts
                     uint32_t s_g[2], s_g8[2], l_g[2], l_g8[2];
-#pragma unroll
-                    for (int b = 0; b < 2; ++b) {
-                        split_scale(fp16_bits_to_float((uint16_t)(sw[b] & 0xFFFFu)), s_g[b], l_g[b]);
-                        split_scale(fp16_bits_to_float((uint16_t)(sw[b] >> 16)), s_g8[b], l_g8[b]);
-                    }
-                    if (BITS == 4) {
-                        const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile_smem + kWeightBytes + kScaleBytes) + g);
-                        uint32_t zg[2], zg8[2];
+                    auto load_scales = [&](int gr) {
+                        const uint2 sc = *(reinterpret_cast<const uint2*>(tile_smem + kWeightBytes + gr * kScaleBytes + g * 16) + (q & 1));
+                        const uint32_t sw[2] = {sc.x, sc.y};
 #pragma unroll
                         for (int b = 0; b < 2; ++b) {
-                            const uint32_t pair = w4_reg_biased(zword, w0 + b);   // (128 + z[row g], 128 + z[row g+8])
-                            zg[b] = __byte_perm(pair, 0, 0x1010);
-                            zg8[b] = __byte_perm(pair, 0, 0x3232);
+                            split_scale(fp16_bits_to_float((uint16_t)(sw[b] & 0xFFFFu)), s_g[b], l_g[b]);
+                            split_scale(fp16_bits_to_float((uint16_t)(sw[b] >> 16)), s_g8[b], l_g8[b]);
                         }
+                    };
+                    if (BITS == 4) {
+                        // This warp's 64 k of the tile lie in one group (group sizes >= 64: group `half` of two, or the
+                        // tile's only one) or in two (group size 32: k-steps 0, 1 and 2, 3).
+                        constexpr int kSubGroups = G == 4 ? 2 : 1;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {              // k-block 4*half + i = MMA k-step i of this operand stage
-                            const uint2 x = *(reinterpret_cast<const uint2*>(tile_smem + ((4 * half + i) * 32 + lane) * 16) + (q & 1));
-                            const uint32_t xs[2] = {x.x, x.y};
+                        for (int sub = 0; sub < kSubGroups; ++sub) {
+                            const int gr = G == 1 ? 0 : G == 2 ? half : 2 * half + sub;
+                            load_scales(gr);
+                            const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile_smem + w4_zero_offset(G, gr)) + g);
+                            uint32_t zg[2], zg8[2];
 #pragma unroll
                             for (int b = 0; b < 2; ++b) {
-                                op[b][4 * i + 0] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 0), zg[b]), s_g[b], l_g[b]);    // row g,   k 0,1
-                                op[b][4 * i + 1] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 2), zg[b]), s_g[b], l_g[b]);    // row g,   k 2,3
-                                op[b][4 * i + 2] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 1), zg8[b]), s_g8[b], l_g8[b]);  // row g+8, k 0,1
-                                op[b][4 * i + 3] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 3), zg8[b]), s_g8[b], l_g8[b]);  // row g+8, k 2,3
+                                const uint32_t pair = w4_reg_biased(zword, w0 + b);   // (128 + z[row g], 128 + z[row g+8])
+                                zg[b] = __byte_perm(pair, 0, 0x1010);
+                                zg8[b] = __byte_perm(pair, 0, 0x3232);
+                            }
+#pragma unroll
+                            for (int i = sub * (4 / kSubGroups); i < (sub + 1) * (4 / kSubGroups); ++i) {   // k-block 4*half + i = MMA k-step i of this operand stage
+                                const uint2 x = *(reinterpret_cast<const uint2*>(tile_smem + ((4 * half + i) * 32 + lane) * 16) + (q & 1));
+                                const uint32_t xs[2] = {x.x, x.y};
+#pragma unroll
+                                for (int b = 0; b < 2; ++b) {
+                                    op[b][4 * i + 0] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 0), zg[b]), s_g[b], l_g[b]);    // row g,   k 0,1
+                                    op[b][4 * i + 1] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 2), zg[b]), s_g[b], l_g[b]);    // row g,   k 2,3
+                                    op[b][4 * i + 2] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 1), zg8[b]), s_g8[b], l_g8[b]);  // row g+8, k 0,1
+                                    op[b][4 * i + 3] = times_scale(bf16x2_sub(w4_reg_biased(xs[b], 3), zg8[b]), s_g8[b], l_g8[b]);  // row g+8, k 2,3
+                                }
                             }
                         }
                     } else {
+                        load_scales(0);
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const uint4 x = *reinterpret_cast<const uint4*>(tile_smem + (((4 * half + i) * 2 + (q & 1)) * 32 + lane) * 16);
@@ -624,7 +643,7 @@ size_t gemm_workspace_bytes(int M, int K, int N) {
 
 namespace {
 
-template <int BITS, int BT>
+template <int BITS, int BT, int G = 1>
 cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, int N, void* workspace, int sm_count,
                       cudaStream_t stream) {
     CUtensorMap map;
@@ -642,8 +661,8 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     const bool seen = dev >= 0 && dev < kMaxDevices;
     if (!seen || !configured_on[dev].load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BITS, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             gemm_smem_bytes(BITS, BT));
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BITS, BT, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             gemm_smem_bytes(BITS, BT, G));
         if (e != cudaSuccess) return e;
         if (seen) configured_on[dev].store(true, std::memory_order_release);
     }
@@ -665,7 +684,7 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(kGemmThreads, 1, 1);
-    cfg.dynamicSmemBytes = gemm_smem_bytes(BITS, BT);
+    cfg.dynamicSmemBytes = gemm_smem_bytes(BITS, BT, G);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see grid_dependency_wait() in the kernel
@@ -673,24 +692,27 @@ cudaError_t launch_bt(const void* blob, const void* a, void* y, int M, int K, in
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     note_whole_sm_launch(stream);
-    return cudaLaunchKernelEx(&cfg, gemm_kernel<BITS, BT>, map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K,
+    return cudaLaunchKernelEx(&cfg, gemm_kernel<BITS, BT, G>, map, static_cast<const uint8_t*>(blob), static_cast<__nv_bfloat16*>(y), M, K,
                               N, ktiles, n_tiles, m_tiles, aligned, static_cast<uint8_t*>(workspace), debug_word());
 }
 
-template <int BITS>
+template <int BITS, int G = 1>
 cudaError_t launch_bits(const void* blob, const void* a, void* y, int M, int K, int N, void* workspace, int sm_count,
                         cudaStream_t stream) {
-    if (M > 128) return launch_bt<BITS, 256>(blob, a, y, M, K, N, workspace, sm_count, stream);
-    if (M > 64) return launch_bt<BITS, 128>(blob, a, y, M, K, N, workspace, sm_count, stream);
-    if (M > 32) return launch_bt<BITS, 64>(blob, a, y, M, K, N, workspace, sm_count, stream);
-    return launch_bt<BITS, 32>(blob, a, y, M, K, N, workspace, sm_count, stream);
+    if (M > 128) return launch_bt<BITS, 256, G>(blob, a, y, M, K, N, workspace, sm_count, stream);
+    if (M > 64) return launch_bt<BITS, 128, G>(blob, a, y, M, K, N, workspace, sm_count, stream);
+    if (M > 32) return launch_bt<BITS, 64, G>(blob, a, y, M, K, N, workspace, sm_count, stream);
+    return launch_bt<BITS, 32, G>(blob, a, y, M, K, N, workspace, sm_count, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_gemm(int bits, const void* blob, const void* a, void* y, int M, int K, int N, void* workspace,
-                        size_t workspace_bytes, int sm_count, cudaStream_t stream) {
+                        size_t workspace_bytes, int sm_count, cudaStream_t stream, int groups) {
     (void)workspace_bytes;
+    if (groups == 2 && bits == 4) return launch_bits<4, 2>(blob, a, y, M, K, N, workspace, sm_count, stream);
+    if (groups == 4 && bits == 4) return launch_bits<4, 4>(blob, a, y, M, K, N, workspace, sm_count, stream);
+    if (groups != 1) return cudaErrorInvalidValue;
     return bits == 4 ? launch_bits<4>(blob, a, y, M, K, N, workspace, sm_count, stream)
                      : launch_bits<8>(blob, a, y, M, K, N, workspace, sm_count, stream);
 }

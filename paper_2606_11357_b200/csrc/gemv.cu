@@ -221,12 +221,14 @@ __device__ __noinline__ bool gather_rows(float4* slot, int count, int M, float4 
 
 }  // namespace
 
-template <int BITS, int MT, bool FULL, bool CL, bool I8>
+// G = groups per tile: 1 for group sizes that are multiples of 128, 2 / 4 for the 4-bit group sizes 64 / 32.
+template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
                    int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes,
                    uint8_t* __restrict__ workspace, uint32_t debug) {
-    constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
+    static_assert(G == 1 || (BITS == 4 && !I8 && !CL && FULL), "several groups per tile: 4-bit, floating-point path, whole SM");
+    constexpr int kTileBytes = tile_bytes(BITS, G);
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
     constexpr int kTok = 8 * MT;
@@ -271,7 +273,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
     float* partials = reinterpret_cast<float*>(workspace + kGemvPartialOffset);
 
-    const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N);
+    const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N) && group_size_fits(blob, G);
 
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kGemvMaxStages);
     const uint32_t seg_full0 = smem_u32(bars + 2 * kGemvMaxStages), seg_free0 = seg_full0 + 16;
@@ -509,8 +511,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 const uint8_t* stage = ring + (size_t)s * stage_bytes;
                 const uint8_t* tile = stage + (size_t)slot * kTileBytes;
 
-                const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
                 if constexpr (I8) {
+                    const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
                     // ---- integer path (1 or 2 tokens): codes x activation pieces on the integer warp MMA ----
                     // The 128 activations of a (token, k-tile) are scaled by 2^(148 - emax) (emax = largest biased
                     // exponent among them), rounded to integers |v| < 2^22 and split into signed bytes
@@ -649,71 +651,78 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                         acc[w][0][3] = fmaf(small_int_to_float(d[w][3]) * col_scale.y, s_g8, acc[w][0][3]);
                     }
                 } else {
-                uint32_t zg[4], zg8[4];
-                if (BITS == 4) {
-                    const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile + kWeightBytes + kScaleBytes) + g);
-                    w4_zero_regs(zword, zg, zg8);
-                }
-                float gacc[4][MT][4];
+                // ---- floating-point path: group after group (one group per tile unless the group size is 64 or 32) ----
 #pragma unroll
-                for (int w = 0; w < 4; ++w)
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) gacc[w][mt][e] = 0.f;
-
-#pragma unroll
-                for (int kb = 0; kb < 8; ++kb) {
-                    uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        av[mt] = ag[mt][kb];
+                for (int gr = 0; gr < G; ++gr) {
+                    const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes + gr * kScaleBytes) + g);
+                    uint32_t zg[4], zg8[4];
+                    if (BITS == 4) {
+                        const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile + w4_zero_offset(G, gr)) + g);
+                        w4_zero_regs(zword, zg, zg8);
                     }
-                    uint4 wv[kVecPerKb];
+                    float gacc[4][MT][4];
 #pragma unroll
-                    for (int h = 0; h < kVecPerKb; ++h)
-                        wv[h] = *reinterpret_cast<const uint4*>(tile + ((size_t)(kb * kVecPerKb + h) * 32 + lane) * 16);
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        uint32_t r0, r1, r2, r3;
-                        if (BITS == 4) {
-                            const uint4 v = wv[0];
-                            const uint32_t x = w == 0 ? v.x : w == 1 ? v.y : w == 2 ? v.z : v.w;
-                            r0 = bf16x2_sub(w4_reg_biased(x, 0), zg[w]);
-                            r1 = bf16x2_sub(w4_reg_biased(x, 1), zg8[w]);
-                            r2 = bf16x2_sub(w4_reg_biased(x, 2), zg[w]);
-                            r3 = bf16x2_sub(w4_reg_biased(x, 3), zg8[w]);
-                        } else {
-                            const uint4 v = wv[(w >> 1) % kVecPerKb];
-                            w8_word_to_regs((w & 1) ? v.z : v.x, r0, r1);
-                            w8_word_to_regs((w & 1) ? v.w : v.y, r2, r3);
-                        }
+                    for (int w = 0; w < 4; ++w)
 #pragma unroll
                         for (int mt = 0; mt < MT; ++mt)
-                            mma_bf16_16816(gacc[w][mt], r0, r1, r2, r3, av[mt].x, av[mt].y);
-                    }
-                    if (has_next) load_ag_kb(next_base, kb);    // this k-block's registers are free: ask for the next tile's
-                }
-                // all shared-memory reads of this tile are done: hand its share of the stage back to the
-                // producer (the last tile of a short chunk also returns the shares of the missing tiles)
-                __syncwarp();
-                if (lane == 0) {
-                    const int tiles_here = min(kR, seg_len - cl * kR);
-                    mbar_arrive_n(empty0 + 8 * s, slot == tiles_here - 1 ? (uint32_t)(kR - tiles_here + 1) : 1u);
-                }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) gacc[w][mt][e] = 0.f;
 
-                // the group's scales, in fp32 (Eq. 1 / Eq. 2 factored per group)
-                const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    const float s_g = fp16_bits_to_float((uint16_t)(sw[w] & 0xFFFFu));
-                    const float s_g8 = fp16_bits_to_float((uint16_t)(sw[w] >> 16));
+                    for (int kb = gr * (8 / G); kb < (gr + 1) * (8 / G); ++kb) {
+                        uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        acc[w][mt][0] = fmaf(s_g, gacc[w][mt][0], acc[w][mt][0]);
-                        acc[w][mt][1] = fmaf(s_g, gacc[w][mt][1], acc[w][mt][1]);
-                        acc[w][mt][2] = fmaf(s_g8, gacc[w][mt][2], acc[w][mt][2]);
-                        acc[w][mt][3] = fmaf(s_g8, gacc[w][mt][3], acc[w][mt][3]);
+                        for (int mt = 0; mt < MT; ++mt) {
+                            av[mt] = ag[mt][kb];
+                        }
+                        uint4 wv[kVecPerKb];
+#pragma unroll
+                        for (int h = 0; h < kVecPerKb; ++h)
+                            wv[h] = *reinterpret_cast<const uint4*>(tile + ((size_t)(kb * kVecPerKb + h) * 32 + lane) * 16);
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            uint32_t r0, r1, r2, r3;
+                            if (BITS == 4) {
+                                const uint4 v = wv[0];
+                                const uint32_t x = w == 0 ? v.x : w == 1 ? v.y : w == 2 ? v.z : v.w;
+                                r0 = bf16x2_sub(w4_reg_biased(x, 0), zg[w]);
+                                r1 = bf16x2_sub(w4_reg_biased(x, 1), zg8[w]);
+                                r2 = bf16x2_sub(w4_reg_biased(x, 2), zg[w]);
+                                r3 = bf16x2_sub(w4_reg_biased(x, 3), zg8[w]);
+                            } else {
+                                const uint4 v = wv[(w >> 1) % kVecPerKb];
+                                w8_word_to_regs((w & 1) ? v.z : v.x, r0, r1);
+                                w8_word_to_regs((w & 1) ? v.w : v.y, r2, r3);
+                            }
+#pragma unroll
+                            for (int mt = 0; mt < MT; ++mt)
+                                mma_bf16_16816(gacc[w][mt], r0, r1, r2, r3, av[mt].x, av[mt].y);
+                        }
+                        if (has_next) load_ag_kb(next_base, kb);    // this k-block's registers are free: ask for the next tile's
+                    }
+                    if (gr == G - 1) {
+                        // all shared-memory reads of this tile are done: hand its share of the stage back to the
+                        // producer (the last tile of a short chunk also returns the shares of the missing tiles)
+                        __syncwarp();
+                        if (lane == 0) {
+                            const int tiles_here = min(kR, seg_len - cl * kR);
+                            mbar_arrive_n(empty0 + 8 * s, slot == tiles_here - 1 ? (uint32_t)(kR - tiles_here + 1) : 1u);
+                        }
+                    }
+
+                    // the group's scales, in fp32 (Eq. 1 / Eq. 2 factored per group)
+                    const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float s_g = fp16_bits_to_float((uint16_t)(sw[w] & 0xFFFFu));
+                        const float s_g8 = fp16_bits_to_float((uint16_t)(sw[w] >> 16));
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            acc[w][mt][0] = fmaf(s_g, gacc[w][mt][0], acc[w][mt][0]);
+                            acc[w][mt][1] = fmaf(s_g, gacc[w][mt][1], acc[w][mt][1]);
+                            acc[w][mt][2] = fmaf(s_g8, gacc[w][mt][2], acc[w][mt][2]);
+                            acc[w][mt][3] = fmaf(s_g8, gacc[w][mt][3], acc[w][mt][3]);
+                        }
                     }
                 }
                 }
@@ -853,8 +862,9 @@ static int max_resident_clusters(int csize, bool full) {
 // 0.7 us later than one that does not, even when launched without clusters, and a cluster launch overlaps less
 // with its neighbours on the stream, so cluster mode has instantiations of its own and is taken only for short
 // ranges, where the hand-over dominates the call.
-GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
+GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     GemvPlan p;
+    p.groups = groups;
     p.strips = (N + kTileN - 1) / kTileN;
     p.ktiles = K / kTileK;
     p.total_tiles = p.strips * p.ktiles;
@@ -905,7 +915,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     // launch next to a plain one does not (about 2.7 us per transition, measured), and in a pass over layers of
     // different sizes that loss is larger than what the short hand-over wins for up to 8 tokens.
     const int one_round = gemv_max_consumers(mt, mt == 2);
-    const bool cluster_ok = mt == 2;
+    const bool cluster_ok = mt == 2 && groups == 1;
     if (p.cluster > 1 && cluster_ok && tiles_per_cta <= 16 && (best_t <= one_round || best_t * 10 <= tiles_per_cta * 11 + 20)) {
         p.grid = p.nclusters * p.cluster;
         tiles_per_cta = best_t;
@@ -918,9 +928,9 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     // warps, deeper ring).  The integer path of 1 and 2 tokens needs a fraction of the instructions; its short ranges
     // gain more from the next GEMV's CTAs sitting beside this one's with their rings already full, long ones
     // amortise the start of the kernel and take the whole SM too.
-    const bool i8_path = M <= kGemvI8MaxM;
-    p.full = mt == 2 || !i8_path || tiles_per_cta * (bits == 4 ? kW4TileBytes : kW8TileBytes) >= kGemvFullFromBytesI8;
-    p.i8 = M <= kGemvI8MaxM && p.cluster == 1;
+    const bool i8_path = M <= kGemvI8MaxM && groups == 1;     // several groups per tile: floating-point path only
+    p.full = mt == 2 || !i8_path || tiles_per_cta * tile_bytes(bits, groups) >= kGemvFullFromBytesI8;
+    p.i8 = i8_path && p.cluster == 1;
     // the integer path leaves the warps waiting for data, not for issue slots: 8 of them keep more tiles in flight
     // (4096x14336, 1 token: 13.7 us with 8 warps, 14.2 us with 12)
     p.consumers = p.i8 && p.full ? 8 : gemv_max_consumers(mt, p.full);
@@ -928,7 +938,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count) {
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
     const int kr = gemv_chunk_tiles(bits);
     // a stage: one bulk copy of kR packed tiles, padded to a multiple of 1 KB
-    p.stage_bytes = kGemvStageBytes;
+    p.stage_bytes = groups == 1 ? kGemvStageBytes : (kr * tile_bytes(bits, groups) + 1023) / 1024 * 1024;
     // cluster mode: one slot per CTA of the cluster for the rows of real tokens (two token rows = 512 bytes)
     p.xslot_bytes = p.cluster > 1 ? ((M + 1) / 2) * 512 : 0;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4 +
@@ -975,20 +985,20 @@ void note_whole_sm_launch(cudaStream_t stream) { note_launch(stream, true); }
 
 // Function attributes belong to one device: set once per device and kernel instantiation.  The flag is atomic: two
 // host threads may both find it unset and both set the attributes, which is harmless.
-template <int BITS, int MT, bool FULL, bool CL, bool I8>
+template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
 static cudaError_t configure_one() {
     static std::atomic<bool> configured_on[kGemvMaxDevices];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     const bool seen = dev >= 0 && dev < kGemvMaxDevices;
     if (seen && configured_on[dev].load(std::memory_order_acquire)) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          FULL ? gemv_smem_budget(MT, FULL) : kGemvSoloSmemBytes);
     if (e != cudaSuccess) return e;
     // Always the largest shared-memory carve-out: a GEMV whose ring happens to be a little smaller would
     // otherwise ask for a smaller split of the SM's memory, and an SM changes its split only when idle, so
     // consecutive GEMVs of different shapes could not share an SM.
-    e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    e = cudaFuncSetAttribute(gemv_stream_kernel<BITS, MT, FULL, CL, I8, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
                              cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     if (seen) configured_on[dev].store(true, std::memory_order_release);
@@ -1004,6 +1014,10 @@ static cudaError_t configure_bits() {
     all(configure_one<BITS, 2, true, false, false>());
     all(configure_one<BITS, 1, false, true, false>());  all(configure_one<BITS, 1, true, true, false>());
     all(configure_one<BITS, 2, true, true, false>());
+    if constexpr (BITS == 4) {
+        all(configure_one<4, 1, true, false, false, 2>()); all(configure_one<4, 2, true, false, false, 2>());
+        all(configure_one<4, 1, true, false, false, 4>()); all(configure_one<4, 2, true, false, false, 4>());
+    }
     return e;
 }
 
@@ -1016,10 +1030,10 @@ cudaError_t configure_gemv_kernels() {
     return e;
 }
 
-template <int BITS, int MT, bool FULL, bool CL, bool I8>
+template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
-    cudaError_t ce = configure_one<BITS, MT, FULL, CL, I8>();
+    cudaError_t ce = configure_one<BITS, MT, FULL, CL, I8, G>();
     if (ce != cudaSuccess) return ce;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.grid, 1, 1);
@@ -1048,7 +1062,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
         attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
         cfg.numAttrs = 2;
     }
-    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8>, static_cast<const uint8_t*>(blob),
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8, G>, static_cast<const uint8_t*>(blob),
                               static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
                               p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace), debug_word());
 }
@@ -1056,6 +1070,16 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
 template <int BITS>
 static cudaError_t launch_bits(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K, int N,
                                void* workspace, cudaStream_t stream) {
+    if constexpr (BITS == 4) {
+        // group sizes 64 and 32: the whole-SM floating-point kernel with two or four groups per tile
+        if (p.groups == 2)
+            return M > 8 ? launch_one<4, 2, true, false, false, 2>(p, blob, a, y, M, K, N, workspace, stream)
+                         : launch_one<4, 1, true, false, false, 2>(p, blob, a, y, M, K, N, workspace, stream);
+        if (p.groups == 4)
+            return M > 8 ? launch_one<4, 2, true, false, false, 4>(p, blob, a, y, M, K, N, workspace, stream)
+                         : launch_one<4, 1, true, false, false, 4>(p, blob, a, y, M, K, N, workspace, stream);
+    }
+    if (p.groups != 1) return cudaErrorInvalidValue;
     // the cluster instructions are compiled only into the instantiations that are launched as clusters
     if (p.cluster > 1) {
         if (M > 8) return launch_one<BITS, 2, true, true, false>(p, blob, a, y, M, K, N, workspace, stream);

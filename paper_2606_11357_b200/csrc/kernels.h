@@ -64,9 +64,10 @@ struct GemvPlan {
     int stage_bytes;   // bytes of one ring stage
     int smem_bytes;
     int strips, ktiles, total_tiles;
+    int groups;        // groups per tile: 1, or 2 / 4 for the 4-bit group sizes 64 / 32
 };
 
-GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count);
+GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups = 1);
 cudaError_t launch_gemv(int bits, const GemvPlan& plan, const void* blob, const void* a, void* y,
                         int M, int K, int N, void* workspace, cudaStream_t stream);
 
@@ -105,6 +106,6 @@ cudaError_t launch_gemv_raw(const RawGemvPlan& plan, const uint32_t* qweight, co
 // Prefill GEMM (tcgen05).  `workspace` starts with the DeviceStatus word.
 size_t gemm_workspace_bytes(int M, int K, int N);
 cudaError_t launch_gemm(int bits, const void* blob, const void* a, void* y, int M, int K, int N,
-                        void* workspace, size_t workspace_bytes, int sm_count, cudaStream_t stream);
+                        void* workspace, size_t workspace_bytes, int sm_count, cudaStream_t stream, int groups = 1);
 
 }  // namespace tf

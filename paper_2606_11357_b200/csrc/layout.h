@@ -19,6 +19,9 @@
 //     byte b of word r holds register 2r + (b>>1), element (b & 1).
 // Scales: fp16 [g][2w+h] for column n0 + 16w + g + 8h  (one 16-byte vector per g).
 // Zeros (W4): uint32 [g]; nibble i (0..3) = column n0 + 16i + g, nibble i+4 = column n0+16i+g+8.
+// Group sizes below the tile's k-extent (W4 only: 64 or 32) put G = 128 / group_size groups into a tile: the
+// tile then carries G scale blocks followed by G zero blocks, group after group along k, and is 160 (G - 1) bytes
+// longer (4416 bytes for group size 64, 4736 for 32).
 #pragma once
 #include <stdint.h>
 
@@ -36,5 +39,18 @@ constexpr int kScaleBytes = 128;
 constexpr int kZeroBytes = 32;
 constexpr int kW4TileBytes = kW4WeightBytes + kScaleBytes + kZeroBytes;   // 4256
 constexpr int kW8TileBytes = kW8WeightBytes + kScaleBytes;                // 8320
+
+// Groups per tile for a legal group size (a multiple of 128 that divides K: one; 64: two; 32: four).
+#ifdef __CUDACC__
+#define TF_HD __host__ __device__
+#else
+#define TF_HD
+#endif
+TF_HD constexpr int groups_per_tile(int group_size) { return group_size >= kTileK ? 1 : kTileK / group_size; }
+// W4 tile with G groups: weights | G scale blocks | G zero blocks.
+TF_HD constexpr int w4_tile_bytes(int G) { return kW4WeightBytes + G * (kScaleBytes + kZeroBytes); }
+TF_HD constexpr int w4_scale_offset(int gr) { return kW4WeightBytes + gr * kScaleBytes; }
+TF_HD constexpr int w4_zero_offset(int G, int gr) { return kW4WeightBytes + G * kScaleBytes + gr * kZeroBytes; }
+TF_HD constexpr int tile_bytes(int bits, int G) { return bits == 4 ? w4_tile_bytes(G) : kW8TileBytes; }
 
 }  // namespace tf

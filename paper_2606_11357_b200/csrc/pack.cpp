@@ -17,8 +17,9 @@ bool legal_shape(int bits, int K, int N, int g) {
     if (bits != 4 && bits != 8) return false;
     if (K < tf::kTileK || K > TF_MAX_DIM || N < 8 || N > TF_MAX_DIM) return false;
     if (N % 8 != 0) return false;
-    if (g <= 0 || g % tf::kTileK != 0 || K % g != 0) return false;
-    return true;
+    if (g <= 0 || K % g != 0) return false;
+    if (g % tf::kTileK == 0) return true;
+    return bits == 4 && (g == 64 || g == 32);      // several groups inside a tile: the 4-bit format only
 }
 
 void write_header(void* out, int bits, int K, int N, int g, size_t total) {
@@ -33,7 +34,7 @@ void write_header(void* out, int bits, int K, int N, int g, size_t total) {
     h.n_padded = (uint32_t)((N + tf::kTileN - 1) / tf::kTileN * tf::kTileN);
     h.strips = h.n_padded / tf::kTileN;
     h.ktiles = (uint32_t)(K / tf::kTileK);
-    h.tile_bytes = bits == 4 ? tf::kW4TileBytes : tf::kW8TileBytes;
+    h.tile_bytes = (uint32_t)tf::tile_bytes(bits, tf::groups_per_tile(g));
     h.tiles_offset = tf::kHeaderBytes;
     h.total_bytes = total;
     memcpy(out, &h, sizeof(h));
@@ -64,7 +65,7 @@ extern "C" __attribute__((visibility("default"))) size_t tf_packed_size(int bits
     if (!legal_shape(bits, K, N, group_size)) return 0;
     size_t strips = (size_t)(N + tf::kTileN - 1) / tf::kTileN;
     size_t ktiles = (size_t)K / tf::kTileK;
-    size_t tile = bits == 4 ? tf::kW4TileBytes : tf::kW8TileBytes;
+    size_t tile = (size_t)tf::tile_bytes(bits, tf::groups_per_tile(group_size));
     return tf::kHeaderBytes + strips * ktiles * tile;
 }
 
@@ -79,11 +80,12 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_pack_awq(const ui
     const size_t row_words = (size_t)N / 8;
     const int strips = (N + tf::kTileN - 1) / tf::kTileN, ktiles = K / tf::kTileK;
     uint8_t* base = static_cast<uint8_t*>(out) + tf::kHeaderBytes;
+    const int G = tf::groups_per_tile(group_size), tile_bytes = tf::w4_tile_bytes(G);
     for (int S = 0; S < strips; ++S) {
         const int n0 = S * tf::kTileN;
         for (int T = 0; T < ktiles; ++T) {
-            const int k0 = T * tf::kTileK, grp = k0 / group_size;
-            uint8_t* tile = base + ((size_t)S * ktiles + T) * tf::kW4TileBytes;
+            const int k0 = T * tf::kTileK;
+            uint8_t* tile = base + ((size_t)S * ktiles + T) * tile_bytes;
             uint32_t* wq = reinterpret_cast<uint32_t*>(tile);
             for (int kb = 0; kb < 8; ++kb)
                 for (int lane = 0; lane < 32; ++lane)
@@ -100,16 +102,19 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_pack_awq(const ui
                         }
                         wq[(kb * 32 + lane) * 4 + w] = word;
                     }
-            write_scales(tile + tf::kW4WeightBytes, scales_fp16, N, grp, n0);
-            uint32_t* zq = reinterpret_cast<uint32_t*>(tile + tf::kW4WeightBytes + tf::kScaleBytes);
-            for (int g = 0; g < 8; ++g) {
-                uint32_t word = 0;
-                for (int i = 0; i < 8; ++i) {
-                    const int n = n0 + 16 * (i & 3) + g + 8 * (i >> 2);
-                    uint32_t code = n < N ? awq_code(qzeros, row_words, grp, n) : 0u;
-                    word |= code << (4 * i);
+            for (int gr = 0; gr < G; ++gr) {                 // the groups that meet this tile, along k
+                const int grp = (k0 + gr * (tf::kTileK / G)) / group_size;
+                write_scales(tile + tf::w4_scale_offset(gr), scales_fp16, N, grp, n0);
+                uint32_t* zq = reinterpret_cast<uint32_t*>(tile + tf::w4_zero_offset(G, gr));
+                for (int g = 0; g < 8; ++g) {
+                    uint32_t word = 0;
+                    for (int i = 0; i < 8; ++i) {
+                        const int n = n0 + 16 * (i & 3) + g + 8 * (i >> 2);
+                        uint32_t code = n < N ? awq_code(qzeros, row_words, grp, n) : 0u;
+                        word |= code << (4 * i);
+                    }
+                    zq[g] = word;
                 }
-                zq[g] = word;
             }
         }
     }

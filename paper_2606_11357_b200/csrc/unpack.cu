@@ -15,9 +15,10 @@ template <int BITS>
 __global__ void unpack_kernel(const uint8_t* __restrict__ blob, uint8_t* __restrict__ q,
                               uint8_t* __restrict__ z, uint16_t* __restrict__ s, int K, int N,
                               int group_size, int ktiles, long long total_items) {
-    constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
-    if (!header_matches(blob, BITS, (uint32_t)K, (uint32_t)N)) return;
+    if (!header_matches(blob, BITS, (uint32_t)K, (uint32_t)N) || header_group_size(blob) != (uint32_t)group_size) return;
+    const int G = groups_per_tile(group_size);                       // groups inside one tile (4-bit, group size 64 / 32)
+    const int kTileBytes = tile_bytes(BITS, G);
     const long long item = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (item >= total_items) return;
     const int w = item & 3, lane = (item >> 2) & 31, kb = (item >> 7) & 7;
@@ -48,13 +49,15 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ blob, uint8_t* __restr
                 if (n < N) q[(size_t)k * N + n] = (uint8_t)val;
             }
     }
-    // metadata: the threads of k-block 0, t == 0 of the first tile of each group write it
-    if (kb == 0 && t == 0 && (k0 % group_size) == 0) {
-        const int grp = k0 / group_size;
-        const uint16_t* sc = reinterpret_cast<const uint16_t*>(tile + kWeightBytes) + g * 8;
+    // metadata: the threads with t == 0 of k-block gr < G write group gr of the tile (of the first tile of a group
+    // that spans several tiles)
+    if (kb < G && t == 0 && (G > 1 || (k0 % group_size) == 0)) {
+        const int gr = kb;
+        const int grp = G > 1 ? T * G + gr : k0 / group_size;
+        const uint16_t* sc = reinterpret_cast<const uint16_t*>(tile + kWeightBytes + gr * kScaleBytes) + g * 8;
         uint32_t zg[4], zg8[4];
         if (BITS == 4) {
-            const uint32_t zword = reinterpret_cast<const uint32_t*>(tile + kWeightBytes + kScaleBytes)[g];
+            const uint32_t zword = reinterpret_cast<const uint32_t*>(tile + w4_zero_offset(G, gr))[g];
             w4_zero_regs(zword, zg, zg8);
         }
 #pragma unroll
@@ -98,22 +101,24 @@ cudaError_t launch_unpack_w8(const void* blob, int8_t* q, uint16_t* s, int K, in
 template <int BITS>
 __global__ void __launch_bounds__(256) dequant_kernel(const uint8_t* __restrict__ blob, __nv_bfloat16* __restrict__ wout, int K,
                                                       int N, int ktiles) {
-    constexpr int kTileBytes = BITS == 4 ? kW4TileBytes : kW8TileBytes;
     constexpr int kWeightBytes = BITS == 4 ? kW4WeightBytes : kW8WeightBytes;
     constexpr int kRow = kTileN + 8;                                 // padded row of the staging tile (bf16 elements)
     __shared__ __align__(16) __nv_bfloat16 stage[kTileK * kRow];
     if (!header_matches(blob, BITS, (uint32_t)K, (uint32_t)N)) return;
+    const int G = groups_per_tile((int)header_group_size(blob));
+    const int kTileBytes = tile_bytes(BITS, G);
     const int tile_id = blockIdx.x;
     const int T = tile_id % ktiles, S = tile_id / ktiles;
     const uint8_t* tile = blob + kHeaderBytes + (size_t)tile_id * kTileBytes;
-    const uint16_t* scales = reinterpret_cast<const uint16_t*>(tile + kWeightBytes);
     for (int item = threadIdx.x; item < 1024; item += 256) {
         const int w = item & 3, lane = (item >> 2) & 31, kb = item >> 7;
         const int g = lane >> 2, t = lane & 3;
+        const int gr = kb / (8 / G);                                 // the group of this k-block inside the tile
+        const uint16_t* scales = reinterpret_cast<const uint16_t*>(tile + kWeightBytes + gr * kScaleBytes);
         uint32_t r[4];
         if (BITS == 4) {
             const uint32_t x = reinterpret_cast<const uint32_t*>(tile)[(kb * 32 + lane) * 4 + w];
-            const uint32_t zword = reinterpret_cast<const uint32_t*>(tile + kWeightBytes + kScaleBytes)[g];
+            const uint32_t zword = reinterpret_cast<const uint32_t*>(tile + w4_zero_offset(G, gr))[g];
             const uint32_t pair = w4_reg_biased(zword, w);                         // (128 + z[row g], 128 + z[row g+8])
             const uint32_t zg = __byte_perm(pair, 0, 0x1010), zg8 = __byte_perm(pair, 0, 0x3232);
 #pragma unroll

@@ -82,10 +82,13 @@ def read_header(blob):
 
 
 def read_blob(blob, bits, K, N, group_size=128):
-    """Decode a blob on the host -> (q [K, Np], z [K/128, Np] or None, s_bits [K/128, Np]) per tile row."""
+    """Decode a blob on the host -> (q [K, Np], z [rows, Np] or None, s_bits [rows, Np]): one metadata row per tile
+    (group sizes that are multiples of 128) or per group (4-bit group sizes 64 and 32: G = 128 / group_size rows per
+    tile, stored as G scale blocks followed by G zero blocks)."""
     strips, ktiles = (N + TILE_N - 1) // TILE_N, K // TILE_K
-    tile_bytes = W4_TILE if bits == 4 else W8_TILE
+    G = 1 if group_size >= TILE_K else TILE_K // group_size
     wbytes = 4096 if bits == 4 else 8192
+    tile_bytes = (4096 + 160 * G) if bits == 4 else W8_TILE
     tiles = blob[HEADER_BYTES:HEADER_BYTES + strips * ktiles * tile_bytes].reshape(strips, ktiles, tile_bytes)
     Np = strips * TILE_N
     q = np.zeros((K, Np), dtype=np.int16)
@@ -111,18 +114,20 @@ def read_blob(blob, bits, K, N, group_size=128):
                 for S in range(strips):
                     for T in range(ktiles):
                         q[T * TILE_K + dk, S * TILE_N + dn] = raw[S, T, kb, w >> 1, lane, 2 * (w & 1) + r, b]
-    sc = np.ascontiguousarray(tiles[:, :, wbytes:wbytes + 128]).view(np.uint16).reshape(strips, ktiles, 8, 4, 2)
-    s = np.zeros((ktiles, Np), dtype=np.uint16)
-    z = np.zeros((ktiles, Np), dtype=np.int16) if bits == 4 else None
+    s = np.zeros((ktiles * G, Np), dtype=np.uint16)
+    z = np.zeros((ktiles * G, Np), dtype=np.int16) if bits == 4 else None
     gg, ww, hh = np.meshgrid(np.arange(8), np.arange(4), np.arange(2), indexing="ij")
     ncol = 16 * ww + gg + 8 * hh
-    if bits == 4:
-        zw = np.ascontiguousarray(tiles[:, :, wbytes + 128:wbytes + 160]).view(np.uint32).reshape(strips, ktiles, 8)
-    for S in range(strips):
-        for T in range(ktiles):
-            s[T, S * TILE_N + ncol] = sc[S, T]
-            if bits == 4:
-                for i in range(8):
-                    z[T, S * TILE_N + 16 * (i & 3) + np.arange(8) + 8 * (i >> 2)] = \
-                        (zw[S, T] >> np.uint32(4 * i)) & np.uint32(0xF)
+    for gr in range(G):
+        sc = np.ascontiguousarray(tiles[:, :, wbytes + 128 * gr:wbytes + 128 * (gr + 1)]).view(np.uint16).reshape(strips, ktiles, 8, 4, 2)
+        if bits == 4:
+            z0 = wbytes + 128 * G + 32 * gr
+            zw = np.ascontiguousarray(tiles[:, :, z0:z0 + 32]).view(np.uint32).reshape(strips, ktiles, 8)
+        for S in range(strips):
+            for T in range(ktiles):
+                s[T * G + gr, S * TILE_N + ncol] = sc[S, T]
+                if bits == 4:
+                    for i in range(8):
+                        z[T * G + gr, S * TILE_N + 16 * (i & 3) + np.arange(8) + 8 * (i >> 2)] = \
+                            (zw[S, T] >> np.uint32(4 * i)) & np.uint32(0xF)
     return q, z, s

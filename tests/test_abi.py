@@ -34,9 +34,10 @@ def test_packed_size():
     assert tf.tf_packed_size(4, 128, 8) == 256 + 4256              # N padded to one strip
     assert tf.tf_packed_size(4, 256, 72) == 256 + 2 * 2 * 4256
     for bad in [(3, 128, 8, 128), (4, 64, 8, 128), (4, 128, 4, 128), (4, 128, 12, 128),
-                (4, 32768 + 128, 8, 128), (4, 128, 32768 + 8, 128), (4, 256, 8, 64), (4, 384, 8, 256)]:
+                (4, 32768 + 128, 8, 128), (4, 128, 32768 + 8, 128), (4, 256, 8, 16), (8, 256, 8, 64), (4, 384, 8, 256)]:
         assert tf.tf_packed_size(*bad) == 0
     assert tf.tf_packed_size(8, 512, 8, 512) > 0                    # per-channel: group_size == K
+    assert tf.tf_packed_size(4, 256, 8, 64) == 256 + 2 * 4416 and tf.tf_packed_size(4, 256, 8, 32) == 256 + 2 * 4736
 
 
 def test_pack_errors_are_codes_not_crashes():

@@ -51,9 +51,59 @@ def test_medium_token_counts_through_the_gemm(M):
 
 
 def test_illegal_group_sizes_are_rejected():
-    assert tf.tf_packed_size(4, 1024, 64, 64) == 0          # below the tile's k-extent
+    assert tf.tf_packed_size(4, 1024, 64, 16) == 0          # below the smallest group size
+    assert tf.tf_packed_size(8, 1024, 64, 64) == 0          # below the tile's k-extent: 4-bit only
     assert tf.tf_packed_size(4, 1024, 64, 384) == 0         # does not divide K
     assert tf.tf_packed_size(8, 1024, 64, 1024) > 0
+
+
+@pytest.mark.parametrize("g", [64, 32])
+@pytest.mark.parametrize("kind,M,K,N", [("gemv", 1, 1024, 512), ("gemv", 2, 4096, 1024), ("gemv", 7, 512, 200), ("gemv", 16, 2048, 1096),
+                                       ("gemv", 3, 4096, 4096), ("gemm", 17, 512, 200), ("gemm", 100, 1024, 328),
+                                       ("gemm", 300, 2048, 1096), ("gemm", 130, 4096, 512)])
+def test_group_sizes_64_and_32(kind, M, K, N, g):
+    """Section 2.2's group-wise quantization with the group sizes below the tile's k-extent: unpack bit-exact, GEMV and
+    GEMM within the stated tolerance, through the *_grouped entry points."""
+    p = wl.make_w4(M, K, N, seed=1400 + M + g, group_size=g)
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    q = torch.full((K, N), 0xEE, dtype=torch.uint8, device="cuda")
+    z = torch.full((K // g, N), 0xEE, dtype=torch.uint8, device="cuda")
+    s = torch.zeros((K // g, N), dtype=torch.float16, device="cuda")
+    tf.tf_unpack_w4(blob, q, z, s, K, N, g)
+    torch.cuda.synchronize()
+    assert np.array_equal(q.cpu().numpy(), orc.unpack_awq(p.qweight))
+    assert np.array_equal(z.cpu().numpy(), orc.unpack_awq(p.qzeros))
+    assert np.array_equal(s.cpu().numpy().view(np.uint16), p.scales_f16.view(np.uint16))
+    a = gu.to_device_bf16(p.a_bf16)
+    guard = 512
+    ybuf = torch.full((guard + M * N + guard,), gu.CANARY, dtype=torch.int16, device="cuda")
+    y = ybuf[guard:guard + M * N].view(torch.bfloat16).view(M, N)
+    op = tf.TF_OP_GEMV_W4A16 if kind == "gemv" else tf.TF_OP_GEMM_W4A16
+    ws = torch.zeros(tf.tf_workspace_size(op, M, K, N), dtype=torch.uint8, device="cuda")
+    fn = tf.tf_gemv_w4a16_grouped if kind == "gemv" else tf.tf_gemm_w4a16_grouped
+    for _ in range(2):
+        fn(blob, a, y, M, K, N, g, ws)
+    assert tf.tf_device_status(ws) == 0
+    raw = ybuf.cpu().numpy().view(np.uint16)
+    assert np.all(raw[:guard] == gu.CANARY) and np.all(raw[guard + M * N:] == gu.CANARY), "write outside y"
+    gu.check_against_oracle(p, raw[guard:guard + M * N].reshape(M, N))
+
+
+def test_group_size_mismatch_is_detected_on_the_device():
+    """A blob packed with group size 64 given to the default entry point (group size 128), and the other way round:
+    the status word says TF_ERR_BLOB and y is untouched."""
+    M, K, N = 2, 512, 256
+    for g_blob, g_call in ((64, 128), (128, 64), (32, 64)):
+        p = wl.make_w4(M, K, N, seed=1500 + g_blob, group_size=g_blob)
+        blob = torch.from_numpy(gu.pack(p)).cuda()
+        big = torch.zeros(tf.tf_packed_size(4, K, N, 32), dtype=torch.uint8, device="cuda")     # room for the largest tiles
+        big[:blob.numel()] = blob
+        a = gu.to_device_bf16(p.a_bf16)
+        y = torch.full((M, N), -2.0, dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, M, K, N), dtype=torch.uint8, device="cuda")
+        tf.tf_gemv_w4a16_grouped(big, a, y, M, K, N, g_call, ws)
+        assert tf.tf_device_status(ws) == 4
+        assert bool((y == -2.0).all())
 
 
 @pytest.mark.parametrize("kind,M,K,N,zero_bytes", [("gemv", 1, 4096, 1024, 1069056), ("gemv", 16, 4096, 4096, 1069056),

@@ -56,6 +56,28 @@ def test_group_size_multiple_of_tile_replicates_metadata():
     assert np.array_equal(s, np.repeat(p.scales_f16.view(np.uint16), 2, axis=0))
 
 
+@pytest.mark.parametrize("g,tile_bytes", [(64, 4416), (32, 4736)])
+@pytest.mark.parametrize("K,N", [(128, 8), (384, 72), (256, 200)])
+def test_w4_group_sizes_below_the_tile(K, N, g, tile_bytes):
+    """Group sizes 64 and 32: a tile carries two or four scale blocks followed by as many zero blocks."""
+    p = wl.make_w4(1, K, N, seed=K + N + g, group_size=g)
+    blob = tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, K, N, g)
+    h = read_header(blob)
+    assert h["group_size"] == g and h["tile_bytes"] == tile_bytes and h["total_bytes"] == blob.nbytes
+    assert blob.nbytes == 256 + (-(-N // 64)) * (K // 128) * tile_bytes == tf.tf_packed_size(4, K, N, g)
+    q, z, s = read_blob(blob, 4, K, N, g)
+    assert np.array_equal(q[:, :N], orc.unpack_awq(p.qweight))
+    assert np.array_equal(z[:, :N], orc.unpack_awq(p.qzeros))
+    assert np.array_equal(s[:, :N], p.scales_f16.view(np.uint16))
+    assert not q[:, N:].any() and not z[:, N:].any() and not s[:, N:].any()
+
+
+def test_group_sizes_that_are_not_legal():
+    assert tf.tf_packed_size(4, 1024, 64, 16) == 0 and tf.tf_packed_size(4, 1024, 64, 48) == 0
+    assert tf.tf_packed_size(8, 1024, 64, 64) == 0           # below the tile: the 4-bit format only
+    assert tf.tf_packed_size(4, 1024, 64, 64) > 0 and tf.tf_packed_size(4, 1024, 64, 32) > 0
+
+
 def test_blob_is_tile_major_and_contiguous_per_strip():
     """Changing one weight changes bytes only inside that weight's tile payload."""
     K, N = 384, 128
