@@ -766,7 +766,9 @@ def run_gpu(args):
 
 def run_gemm_sweep(args):
     """Shape stability of the prefill GEMM (the paper's kernel evaluation, Section 5.1: M swept in steps of 256 over
-    two shapes with K and N swapped).  Prints one JSON object with TFLOP/s per (shape, M)."""
+    two shapes with K and N swapped), preceded by the token counts between the decode and the prefill range, which
+    take the same entry point with token tiles of 32 / 64 / 128.  Prints one JSON object with us and TFLOP/s per
+    (shape, M)."""
     import torch
     from paper_2606_11357_b200 import binding as tf
     from paper_2606_11357_b200 import workloads as wl
@@ -776,7 +778,7 @@ def run_gemm_sweep(args):
     for (K, N) in ((4096, 14336), (14336, 4096)):
         p = wl.make_w4(1, K, N, seed=11)
         blob = torch.from_numpy(tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, K, N)).to(dev)
-        for M in range(256, 4097, 256):
+        for M in (17, 32, 64, 128, 192) + tuple(range(256, 4097, 256)):       # below 256: the narrower token tiles
             a = torch.randn((M, K), device=dev).to(torch.bfloat16)
             y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
             ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, M, K, N), dtype=torch.uint8, device=dev)
