@@ -44,7 +44,6 @@
 
 namespace tf {
 
-
 namespace {
 
 // Integer warp MMA: D(16x8, s32) += A(16x32, s8) . B(32x8, s8).  Thread (g, t): a0 = row g, k 4t..4t+3; a1 = row g+8;
@@ -225,7 +224,7 @@ __device__ __noinline__ bool gather_rows(float4* slot, int count, int M, float4 
 template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
 gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
-                   int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes,
+                   int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes, int nred,
                    uint8_t* __restrict__ workspace, uint32_t debug) {
     static_assert(G == 1 || (BITS == 4 && !I8 && !CL && FULL), "several groups per tile: 4-bit, floating-point path, whole SM");
     constexpr int kTileBytes = tile_bytes(BITS, G);
@@ -247,7 +246,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     const int nconsumers = (blockDim.x >> 5) - 2;
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
     // xred [csize][xslot]: in cluster mode, the partials other CTAs of the cluster send to the finisher of a strip
-    uint8_t* xred = smem + kGemvBarrierBytes + nconsumers * kRedWarp * 4;
+    uint8_t* xred = smem + kGemvBarrierBytes + nred * nconsumers * kRedWarp * 4;
     // pscr [consumers][1 KB]: integer path, a warp's activation pieces of the tile it works on
     uint32_t* pscr = reinterpret_cast<uint32_t*>(xred + ((CL && csize > 1 ? csize * xslot_bytes : 0) + 1023) / 1024 * 1024);
     uint8_t* ring = reinterpret_cast<uint8_t*>(pscr) + (I8 ? nconsumers * 1024 : 0);
@@ -283,8 +282,10 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             mbar_init(empty0 + 8 * s, kR);       // every tile of a chunk is released by its consumer warp
             stage_tag[s] = 0xFFFFFFFFu;
         }
-        mbar_init(seg_full0, nconsumers);               // every consumer warp has dropped its partial
-        mbar_init(seg_free0, 1);                        // the reducer has read them
+        for (int b = 0; b < 2; ++b) {                   // one pair per partial-sum buffer (nred = 1 or 2)
+            mbar_init(seg_full0 + 8 * b, nconsumers);   // every consumer warp has dropped its partial
+            mbar_init(seg_free0 + 8 * b, 1);            // the reducer has read them
+        }
         abort_flag[0] = 0;
         abort_flag[1] = wait_limit_kcycles(debug);
         mbar_init_fence();
@@ -373,14 +374,16 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     if (!ok) break;
                 }
 
-                ok = mbar_wait(seg_full0, sidx & 1, abort_flag, 0x400);
+                // segment sidx goes through buffer sidx % nred, in that buffer's use number sidx / nred
+                const int rb = nred == 2 ? (sidx & 1) : 0, ru = nred == 2 ? (sidx >> 1) : sidx;
+                ok = mbar_wait(seg_full0 + 8 * rb, ru & 1, abort_flag, 0x400);
                 if (!ok) break;
                 // sum = partial of warp 0 + warp 1 + ... (fixed order); rows of tokens >= M hold zeros
                 float4 sum[kVec];
 #pragma unroll
                 for (int e = 0; e < kVec; ++e) sum[e] = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int w = 0; w < nconsumers; ++w) {
-                    const float4* src = reinterpret_cast<const float4*>(red + (size_t)w * kRedWarp) + lane;
+                    const float4* src = reinterpret_cast<const float4*>(red + (size_t)(rb * nconsumers + w) * kRedWarp) + lane;
 #pragma unroll
                     for (int e = 0; e < kVec; ++e) {
                         const float4 v = src[32 * e];
@@ -388,7 +391,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(seg_free0);                  // consumers may reuse the buffer
+                if (lane == 0) mbar_arrive(seg_free0 + 8 * rb);         // consumers may reuse the buffer
 
                 if (whole || finisher) {
                     // fixed order: the other contributors in CTA order, then this CTA
@@ -467,10 +470,11 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 for (int kb = 0; kb < 8; ++kb) load_ag_kb(base, kb);
             }
         }
+        int T0 = t0 % ktiles;                           // k-tile index at which the current segment starts (0 after the first)
+        int j = cw;                                     // this warp's next tile, as a local index of the CTA's range
         while (i < ntiles && !aborted) {
-            const int tile0 = t0 + i;
-            const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
             const int seg_len = min(ntiles - i, ktiles - T0);
+            T0 = 0;
 
             float acc[4][MT][4];
 #pragma unroll
@@ -480,8 +484,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[w][mt][e] = 0.f;
 
-            // first local tile index >= i handled by this warp
-            int j = i + ((cw - (i % nconsumers)) + nconsumers) % nconsumers;
+            // the warp's tiles come every nconsumers-th tile of the range, whatever segment they fall into
             for (; j < i + seg_len; j += nconsumers) {
                 const int lj = j - i, cl = lj / kR, slot = lj - cl * kR;
                 const int cg = chunk_base + cl;
@@ -730,8 +733,11 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             if (aborted) break;
 
             // ---- drop this warp's partial of the segment for the reducer and move on ---------------------------
-            if (!mbar_wait(seg_free0, (sidx & 1) ^ 1, abort_flag, 0x300)) { aborted = true; break; }   // previous segment read
-            float* mine = red + (size_t)cw * kRedWarp;                          // [token][n]
+            // With two buffers a warp that is a segment ahead of the slowest warp does not wait for it: a segment's
+            // partials go to buffer sidx % nred, which the reducer must have read nred segments ago.
+            const int rb = nred == 2 ? (sidx & 1) : 0, ru = nred == 2 ? (sidx >> 1) : sidx;
+            if (!mbar_wait(seg_free0 + 8 * rb, (ru & 1) ^ 1, abort_flag, 0x300)) { aborted = true; break; }
+            float* mine = red + (size_t)(rb * nconsumers + cw) * kRedWarp;      // [token][n]
             if constexpr (I8) {
                 // columns 3m .. 3m+2 are the pieces of token m, already on a common scale: add them up across the four
                 // threads of a row (fixed order) and leave tokens 0, 1 where the bf16 path has them (t = 0)
@@ -761,7 +767,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     mine[(tok + 1) * kTileN + 16 * w + g + 8] = acc[w][mt][3];
                 }
             __syncwarp();
-            if (lane == 0) mbar_arrive(seg_full0);
+            if (lane == 0) mbar_arrive(seg_full0 + 8 * rb);
             chunk_base += (seg_len + kR - 1) / kR;
             i += seg_len;
             ++sidx;
@@ -941,7 +947,10 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     p.stage_bytes = groups == 1 ? kGemvStageBytes : (kr * tile_bytes(bits, groups) + 1023) / 1024 * 1024;
     // cluster mode: one slot per CTA of the cluster for the rows of real tokens (two token rows = 512 bytes)
     p.xslot_bytes = p.cluster > 1 ? ((M + 1) / 2) * 512 : 0;
-    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.consumers * 8 * mt * kTileN * 4 +
+    // two buffers for the consumer warps' partial sums where the whole SM is taken (a boundary between strips then
+    // costs a fast warp nothing; measured below), one in the half-SM form, where the second would cost a ring stage
+    p.nred = p.full ? 2 : 1;
+    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.nred * p.consumers * 8 * mt * kTileN * 4 +
                       (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (p.i8 ? p.consumers * 1024 : 0);
     int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
     if (stages > kGemvMaxStages) stages = kGemvMaxStages;
@@ -1064,7 +1073,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     }
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8, G>, static_cast<const uint8_t*>(blob),
                               static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
-                              p.cluster, p.nclusters, p.xslot_bytes, static_cast<uint8_t*>(workspace), debug_word());
+                              p.cluster, p.nclusters, p.xslot_bytes, p.nred, static_cast<uint8_t*>(workspace), debug_word());
 }
 
 template <int BITS>

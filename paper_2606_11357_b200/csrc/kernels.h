@@ -64,6 +64,7 @@ struct GemvPlan {
     int stage_bytes;   // bytes of one ring stage
     int smem_bytes;
     int strips, ktiles, total_tiles;
+    int nred;          // buffers for the consumer warps' partial sums of a strip segment (1 or 2)
     int groups;        // groups per tile: 1, or 2 / 4 for the 4-bit group sizes 64 / 32
 };
 
