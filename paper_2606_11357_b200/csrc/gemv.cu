@@ -249,7 +249,9 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     uint8_t* xred = smem + kGemvBarrierBytes + nred * nconsumers * kRedWarp * 4;
     // pscr [consumers][1 KB]: integer path, a warp's activation pieces of the tile it works on
     uint32_t* pscr = reinterpret_cast<uint32_t*>(xred + ((CL && csize > 1 ? csize * xslot_bytes : 0) + 1023) / 1024 * 1024);
-    uint8_t* ring = reinterpret_cast<uint8_t*>(pscr) + (I8 ? nconsumers * 1024 : 0);
+    // abuf [consumers][2][16 rows of kActRowBytes]: 9..16 tokens, a warp's activations of the tile it works on and of its next one
+    uint8_t* abuf = reinterpret_cast<uint8_t*>(pscr) + (I8 ? nconsumers * 1024 : 0);
+    uint8_t* ring = abuf + (MT == 2 ? nconsumers * kGemvActWarpBytes : 0);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
@@ -436,7 +438,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         // before the dependency wait; up to 8 tokens the fragments of the NEXT tile are then requested as soon as a
         // k-block of the current tile has used its registers, so their L2 latency runs under the rest of the tile.
         uint2 araw[2];                                  // integer path: token m, k = 128 T + 4 lane .. +3
-        uint2 ag[!I8 ? MT : 1][!I8 ? 8 : 1];            // token g (+8): k = 128 T + 16 kb + 4t .. +3
+        constexpr bool kRegActs = !I8 && MT == 1;       // floating-point path up to 8 tokens: fragments in registers
+        uint2 ag[1][kRegActs ? 8 : 1];                  // token g: k = 128 T + 16 kb + 4t .. +3
         int T_act = (t0 + cw) % ktiles;                 // k-tile index of this warp's current tile (one division per kernel)
         auto load_araw = [&](const __nv_bfloat16* base) {
 #pragma unroll
@@ -446,22 +449,40 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             }
         };
         auto load_ag_kb = [&](const __nv_bfloat16* base, int kb) {
-#pragma unroll
-            for (int mt = 0; mt < (!I8 ? MT : 1); ++mt)
-                if (g + 8 * mt < M)
-                    ag[mt][!I8 ? kb : 0] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)(g + 8 * mt) * K + 4 * t + 16 * kb));
+            if (g < M) ag[0][kRegActs ? kb : 0] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)g * K + 4 * t + 16 * kb));
         };
         grid_dependency_wait();                         // the activations belong to earlier kernels until now
-        if constexpr (!I8) {
+        if constexpr (kRegActs) {
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                for (int kb = 0; kb < 8; ++kb) ag[mt][kb] = make_uint2(0u, 0u);
+            for (int kb = 0; kb < 8; ++kb) ag[0][kb] = make_uint2(0u, 0u);
         }
-        // One tile ahead only for up to 8 tokens: with 16 tokens the fragments are 32 registers that would stay live
-        // across the whole tile, and the kernel is slower with them (measured: 62.1 against 55.7 us over the four
-        // layer shapes); there a tile's activations are requested when the tile begins, before the wait for its weights.
+        // Up to 8 tokens the fragments are held in registers, one tile ahead.  With 9..16 tokens they would be 32
+        // registers live across the whole tile (measured slower), and a tile that asks for them when it begins waits a
+        // whole trip to the L2 for its first MMA; there the warp copies the 16 x 128 activations of its NEXT tile into
+        // its own shared-memory buffer with cp.async (no registers, from the L2) while it works on the current one, and
+        // takes each fragment from there with one 8-byte load.  Rows are 288 bytes apart, so the eight token rows of a
+        // fragment load fall into different banks (two wavefronts for 256 bytes, the minimum).
         constexpr bool kAhead = MT == 1;
+        constexpr bool kStaged = MT == 2;
+        uint8_t* my_abuf = abuf + (size_t)cw * kGemvActWarpBytes;
+        auto stage_acts = [&](const __nv_bfloat16* base, int buf) {     // one k-tile of activations, rows < M only
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int chunk = lane + 32 * c, row = chunk >> 4, col = chunk & 15;
+                if (row < M) cp_async_16(smem_u32(my_abuf + buf * kGemvActBufBytes + row * kGemvActRowBytes + col * 16), base + (size_t)row * K + col * 8);
+            }
+            cp_async_commit();
+        };
+        if constexpr (kStaged) {
+            // rows of tokens >= M stay zero in both buffers for the whole kernel
+            for (int idx = lane; idx < 2 * 16 * (kGemvActRowBytes / 16); idx += 32) {
+                const int row = (idx / (kGemvActRowBytes / 16)) & 15;
+                if (row >= M) reinterpret_cast<uint4*>(my_abuf)[idx] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            __syncwarp();
+            if (cw < ntiles) stage_acts(a_glob + (size_t)T_act * kTileK, 0);
+        }
+        int abuf_cur = 0;
         if (kAhead && cw < ntiles) {
             const __nv_bfloat16* base = a_glob + (size_t)T_act * kTileK;
             if constexpr (I8) load_araw(base);
@@ -493,15 +514,21 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
                 const int s = s_cur;
                 const bool has_next = kAhead && j + nconsumers < ntiles;
-                if constexpr (!kAhead) {
-                    const __nv_bfloat16* base = a_glob + (size_t)T_act * kTileK;
-#pragma unroll
-                    for (int kb = 0; kb < 8; ++kb) load_ag_kb(base, kb);
-                }
                 int T_nx = T_act + nconsumers;                  // the warp's next tile is nconsumers tiles further along K
                 while (T_nx >= ktiles) T_nx -= ktiles;
                 T_act = T_nx;
                 const __nv_bfloat16* next_base = a_glob + (size_t)T_nx * kTileK;
+                const uint8_t* acts = my_abuf + abuf_cur * kGemvActBufBytes;       // 9..16 tokens: this tile's activations
+                if constexpr (kStaged) {
+                    if (j + nconsumers < ntiles) {
+                        stage_acts(next_base, abuf_cur ^ 1);     // the next tile's, into the other buffer
+                        cp_async_wait<1>();                      // everything but that last group has landed
+                    } else {
+                        cp_async_wait<0>();
+                    }
+                    __syncwarp();                                // every lane's copies are visible to the warp
+                    abuf_cur ^= 1;
+                }
                 if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
                     const long long t_begin = clock64();
                     while (stage_tag[s] != (uint32_t)cg && !aborted) {
@@ -676,7 +703,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                         uint2 av[MT];                              // token g (+8): k = 16kb + 4t .. +3
 #pragma unroll
                         for (int mt = 0; mt < MT; ++mt) {
-                            av[mt] = ag[mt][kb];
+                            if constexpr (kStaged) av[mt] = *reinterpret_cast<const uint2*>(acts + (g + 8 * mt) * kGemvActRowBytes + kb * 32 + t * 8);
+                            else av[mt] = ag[0][kRegActs ? kb : 0];
                         }
                         uint4 wv[kVecPerKb];
 #pragma unroll
@@ -951,7 +979,8 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // costs a fast warp nothing; measured below), one in the half-SM form, where the second would cost a ring stage
     p.nred = p.full ? 2 : 1;
     const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.nred * p.consumers * 8 * mt * kTileN * 4 +
-                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (p.i8 ? p.consumers * 1024 : 0);
+                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (p.i8 ? p.consumers * 1024 : 0) +
+                      (mt == 2 ? p.consumers * kGemvActWarpBytes : 0);
     int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
     if (stages > kGemvMaxStages) stages = kGemvMaxStages;
     // no more stages than the range has chunks

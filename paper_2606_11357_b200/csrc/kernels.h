@@ -36,6 +36,10 @@ constexpr int kGemvMaxContrib = 320;          // CTAs that can share one strip (
 __host__ __device__ constexpr int gemv_chunk_tiles(int bits) { return bits == 4 ? 4 : 2; }
 constexpr int kGemvStageBytes = 17408;        // 17 x 1024 >= 4 x 4256 and >= 2 x 8320
 constexpr int kGemvMaxM = 16;
+// 9..16 tokens: per consumer warp two buffers of 16 token rows x 128 k of activations, rows padded to 288 bytes
+constexpr int kGemvActRowBytes = 288;
+constexpr int kGemvActBufBytes = 16 * kGemvActRowBytes;
+constexpr int kGemvActWarpBytes = 2 * kGemvActBufBytes;
 constexpr int kGemvI8MaxM = 2;                // up to this many tokens the GEMV runs on the integer warp MMA (4-bit and int8 weights)
 constexpr int kGemvMaxGrid = 256;             // CTAs (one per SM); sizes the partial-sum area
 // Workspace layout, shared with the GEMM so that one workspace serves every call of a stream:
