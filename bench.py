@@ -800,6 +800,83 @@ def run_gemm_sweep(args):
     return 0
 
 
+def gather_columns(y_local, counts):
+    """All-gather of column shards: rank r holds y_local [M, counts[r]]; returns y [M, sum(counts)] on every rank.
+    The only exchange of the column-parallel arrangement (Section 4.4: distinct output columns per worker, shared
+    activations, no partial sums between workers).  NCCL on GPUs, gloo in the CPU test."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return y_local
+    world, M, width = dist.get_world_size(), y_local.shape[0], max(counts)
+    padded = torch.zeros((M, width), dtype=y_local.dtype, device=y_local.device)
+    padded[:, :y_local.shape[1]] = y_local
+    out = [torch.empty((M, width), dtype=y_local.dtype, device=y_local.device) for _ in range(world)]
+    dist.all_gather(out, padded)
+    return torch.cat([out[r][:, :counts[r]] for r in range(world)], dim=1)
+
+
+def run_column_parallel(args):
+    """One decode pass over the four layer shapes with every matrix sharded by columns over the ranks (Section 4.4):
+    each rank packs its shard out of the full blob (tf_pack_shard), multiplies the full activations into it
+    (tf_gemv_w4a16 with N = its column count) and the results are all-gathered.  Strong scaling: the total work is
+    fixed.  Prints one JSON line.  On one GPU the shard is the whole matrix and the gather is the identity."""
+    import torch
+    from paper_2606_11357_b200 import binding as tf
+    from paper_2606_11357_b200 import workloads as wl
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank % torch.cuda.device_count())
+    dev = torch.device("cuda", torch.cuda.current_device())
+    init_dist("nccl")
+    M = args.profile_m or 1
+    stream = torch.cuda.current_stream()
+    ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, 16, 4096, 4096), dtype=torch.uint8, device=dev)
+    layers, total_bytes = [], 0
+    for (K, N) in wl.LLAMA3_8B_SHAPES:
+        prob = wl.config1(M, K, N)
+        full = tf.tf_pack_awq(prob.qweight, prob.scales_f16, prob.qzeros, K, N)
+        counts = [tf.tf_shard_columns(N, r, world)[1] for r in range(world)]
+        shard = torch.from_numpy(tf.tf_pack_shard(full, rank, world)).to(dev)
+        copies = [shard] + [shard.clone() for _ in range(int(300e6 // max(shard.numel(), 1)) + 1)]   # beyond L2 in rotation
+        a = torch.from_numpy(prob.a_bf16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+        y_local = torch.empty((M, counts[rank]), dtype=torch.bfloat16, device=dev)
+        layers.append((K, N, counts, copies, a, y_local))
+        total_bytes += gemv_algorithmic_bytes(4, M, K, N)
+    it = {"i": 0}
+
+    def step():
+        it["i"] += 1
+        outs = []
+        for (K, N, counts, copies, a, y_local) in layers:
+            tf.tf_gemv_w4a16(copies[it["i"] % len(copies)], a, y_local, M, K, counts[rank], ws)
+            outs.append(gather_columns(y_local, counts))
+        return outs
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = min(args.steps, 2000)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), dev) / steps
+    if tf.tf_device_status(ws) != 0:
+        raise SystemExit("device status word reports an error")
+    if rank == 0:
+        print(json.dumps({"mode": "column_parallel", "metric": "W4A16 GEMV GB/s", "value": total_bytes / (ms * 1e-3) / 1e9,
+                          "unit": "GB/s", "n_gpus": world, "steps": steps, "ms_per_step": ms, "scaling": "strong",
+                          "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                          "config": {"workload": f"Llama-3-8B layer shapes at M = {M}, every matrix sharded by columns over the ranks, "
+                                                 "results all-gathered; calls issued one by one",
+                                     "columns_per_rank": {f"{K}x{N}": counts for (K, N, counts, _, _, _) in layers}}}), flush=True)
+    return 0
+
+
 def run_profile_case(args):
     """A handful of launches of one kernel on one seeded case, for `ncu` captures (prints no bench line)."""
     import torch
@@ -849,10 +926,14 @@ def main(argv=None):
                     help="run --steps launches of one kernel on one case and exit (for ncu captures)")
     ap.add_argument("--profile-m", type=int, default=0, help="token count for --profile-case")
     ap.add_argument("--profile-shape", default="", help="KxN of a config-1 layer shape for --profile-case gemv_w4 (default 4096x14336)")
+    ap.add_argument("--column-parallel", action="store_true",
+                    help="decode pass with every matrix sharded by columns over the ranks and the results all-gathered (--profile-m tokens)")
     ap.add_argument("--gemm-sweep", action="store_true", help="time the W4A16 GEMM for M = 256..4096 on two K/N-swapped shapes")
     args = ap.parse_args(argv)
     if args.gemm_sweep:
         return run_gemm_sweep(args)
+    if args.column_parallel:
+        return run_column_parallel(args)
     if args.profile_case:
         return run_profile_case(args)
     if args.warmup < 3:

@@ -165,6 +165,22 @@ tf_status tf_unpack_w8(const void* packed, int8_t* q, uint16_t* s_fp16,
 tf_status tf_pack_concat(const void* const* parts, int count, void* out, size_t out_bytes);
 
 /*
+ * Column-parallel sharding over several GPUs (Section 4.4: every worker owns distinct output columns, the
+ * activations are shared, no partial sums travel between workers).
+ * tf_shard_columns: the column range [n_begin, n_begin + n_count) of part `part` of `parts` when the N columns are
+ *   dealt out in whole strips of TF_TILE_N (the last part takes the ragged end); pure arithmetic.
+ * tf_pack_shard: the blob of that column range, cut out of the blob of the whole matrix (host): byte for byte what
+ *   the packer gives for the column-sliced inputs.  Each GPU then calls tf_gemv_* / tf_gemm_* with N = n_count on
+ *   its shard and the full activations, and writes y[:, n_begin : n_begin + n_count]; the only exchange is an
+ *   all-gather of the results (NCCL), done by the caller.
+ *   out_bytes at least tf_packed_size(bits, K, n_count, group_size).  `out` must not overlap `packed`.
+ * Errors: TF_ERR_NULL, TF_ERR_BLOB (not a valid blob), TF_ERR_SHAPE (part outside 0..parts-1, more parts than
+ *         strips), TF_ERR_WORKSPACE (out_bytes too small).
+ */
+tf_status tf_shard_columns(int N, int part, int parts, int* n_begin, int* n_count);
+tf_status tf_pack_shard(const void* packed, int part, int parts, void* out, size_t out_bytes);
+
+/*
  * Ablation baseline (Sections 4.1 and 5.5): dequantize the whole matrix into global memory, to be
  * multiplied by a separate full-precision kernel -- the arrangement the fused kernels replace.
  *   packed   device blob; bits = 4 or 8 must match it.

@@ -24,7 +24,7 @@ EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
            "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan", "tf_debug_inject", "tf_gemv_w4a16_static_status",
-           "tf_gemv_w4a16_grouped", "tf_gemm_w4a16_grouped")
+           "tf_gemv_w4a16_grouped", "tf_gemm_w4a16_grouped", "tf_shard_columns", "tf_pack_shard")
 
 
 class TileFuseError(RuntimeError):
@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.tf_pack_awq.restype, L.tf_pack_awq.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, vp, c_size]
         L.tf_pack_w8.restype, L.tf_pack_w8.argtypes = c_int, [vp, vp, c_int, c_int, c_int, vp, c_size]
         L.tf_pack_concat.restype, L.tf_pack_concat.argtypes = c_int, [vp, c_int, vp, c_size]
+        L.tf_shard_columns.restype, L.tf_shard_columns.argtypes = c_int, [c_int, c_int, c_int, vp, vp]
+        L.tf_pack_shard.restype, L.tf_pack_shard.argtypes = c_int, [vp, c_int, c_int, vp, c_size]
         L.tf_unpack_w4.restype, L.tf_unpack_w4.argtypes = c_int, [vp, vp, vp, vp, c_int, c_int, c_int, vp]
         L.tf_unpack_w8.restype, L.tf_unpack_w8.argtypes = c_int, [vp, vp, vp, c_int, c_int, c_int, vp]
         for name in ("tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16"):
@@ -139,6 +141,25 @@ def tf_pack_concat(parts, out=None) -> np.ndarray:
         out = np.empty(256 + max(payload, 0), dtype=np.uint8)
     ptrs = (ctypes.c_void_p * max(len(parts), 1))(*[p.ctypes.data for p in parts])
     _check("tf_pack_concat", lib().tf_pack_concat(ctypes.cast(ptrs, ctypes.c_void_p), len(parts), out.ctypes.data, out.nbytes))
+    return out
+
+
+def tf_shard_columns(N: int, part: int, parts: int):
+    """(n_begin, n_count) of column shard `part` of `parts` (whole strips of 64 columns)."""
+    b, c = ctypes.c_int(0), ctypes.c_int(0)
+    _check("tf_shard_columns", lib().tf_shard_columns(N, part, parts, ctypes.byref(b), ctypes.byref(c)))
+    return b.value, c.value
+
+
+def tf_pack_shard(packed, part: int, parts: int, out=None) -> np.ndarray:
+    """The blob of column shard `part` of `parts`, cut out of the blob of the whole matrix (host arrays)."""
+    packed = _host(packed, np.uint8)
+    hdr = np.frombuffer(packed[:48].tobytes(), dtype=np.uint32)
+    bits, K, N, g = int(hdr[2]), int(hdr[3]), int(hdr[4]), int(hdr[5])
+    _, count = tf_shard_columns(N, part, parts)
+    if out is None:
+        out = np.empty(tf_packed_size(bits, K, count, g), dtype=np.uint8)
+    _check("tf_pack_shard", lib().tf_pack_shard(packed.ctypes.data, part, parts, out.ctypes.data, out.nbytes))
     return out
 
 

@@ -191,3 +191,37 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_pack_concat(const
     write_header(out, (int)first.bits, (int)first.K, (int)n_total, (int)first.group_size, total);
     return TF_OK;
 }
+
+// Column-parallel sharding (Section 4.4: every worker owns distinct output columns, the activation vector is shared,
+// no partial sums travel between workers).  Tiles are stored strip after strip, so the blob of a column range that
+// starts and ends on strip boundaries is a contiguous byte range of the full blob plus a header of its own.
+extern "C" __attribute__((visibility("default"))) tf_status tf_shard_columns(int N, int part, int parts, int* n_begin, int* n_count) {
+    if (!n_begin || !n_count) return TF_ERR_NULL;
+    if (N < 8 || N > TF_MAX_DIM || N % 8 != 0 || parts < 1 || part < 0 || part >= parts) return TF_ERR_SHAPE;
+    const int strips = (N + tf::kTileN - 1) / tf::kTileN;
+    if (parts > strips) return TF_ERR_SHAPE;                       // every part must own at least one strip
+    const int s0 = (int)(((long long)part * strips) / parts), s1 = (int)(((long long)(part + 1) * strips) / parts);
+    const int b = s0 * tf::kTileN, e = s1 * tf::kTileN < N ? s1 * tf::kTileN : N;
+    *n_begin = b;
+    *n_count = e - b;
+    return TF_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_pack_shard(const void* packed, int part, int parts, void* out, size_t out_bytes) {
+    if (!packed || !out) return TF_ERR_NULL;
+    tf_blob_header h;
+    memcpy(&h, packed, sizeof(h));
+    if (h.magic != tf::kMagic || h.version != tf::kBlobVersion) return TF_ERR_BLOB;
+    if (h.total_bytes == 0 || h.total_bytes != tf_packed_size((int)h.bits, (int)h.K, (int)h.N, (int)h.group_size)) return TF_ERR_BLOB;
+    int n0 = 0, nc = 0;
+    tf_status st = tf_shard_columns((int)h.N, part, parts, &n0, &nc);
+    if (st != TF_OK) return st;
+    const size_t total = tf_packed_size((int)h.bits, (int)h.K, nc, (int)h.group_size);
+    if (total == 0) return TF_ERR_SHAPE;
+    if (out_bytes < total) return TF_ERR_WORKSPACE;
+    const size_t strip_bytes = (size_t)h.ktiles * h.tile_bytes;
+    memcpy(static_cast<uint8_t*>(out) + tf::kHeaderBytes,
+           static_cast<const uint8_t*>(packed) + tf::kHeaderBytes + (size_t)(n0 / tf::kTileN) * strip_bytes, total - tf::kHeaderBytes);
+    write_header(out, (int)h.bits, (int)h.K, nc, (int)h.group_size, total);
+    return TF_OK;
+}

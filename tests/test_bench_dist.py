@@ -32,6 +32,29 @@ def test_two_ranks_gloo():
     assert out[0] == out[1] == (11.0, 4.5)
 
 
+def _gather_worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    bench.init_dist("gloo")
+    from paper_2606_11357_b200 import binding as tf
+    N, M = 200, 3                                           # four strips, the last one ragged: shards of 128 and 72 columns
+    counts = [tf.tf_shard_columns(N, r, world)[1] for r in range(world)]
+    begin = tf.tf_shard_columns(N, rank, world)[0]
+    full = torch.arange(M * N, dtype=torch.float32).reshape(M, N)
+    y = bench.gather_columns(full[:, begin:begin + counts[rank]].contiguous(), counts)
+    out[rank] = (counts, bool(torch.equal(y, full)))
+    dist.destroy_process_group()
+
+
+def test_column_shards_gather_back_on_two_gloo_ranks():
+    """The one exchange of the column-parallel arrangement: ragged column shards all-gathered into the full result."""
+    world, port = 2, 29733
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_gather_worker, args=(world, port, out), nprocs=world, join=True)
+    assert out[0] == out[1] == ([128, 72], True)
+
+
 def test_single_process_passthrough():
     assert bench.max_over_ranks(3.25) == 3.25 and bench.sum_over_ranks(2.0) == 2.0
 

@@ -320,3 +320,23 @@ def test_same_sign_inputs_gemm_stays_within_two_roundings(bits, M, K, N):
     err = np.abs(bf16_bits_to_f64(y_bits) - y_ref)
     assert np.all(err <= 2.0 * 2.0 ** -8 * bound + 1e-5)
     assert float(np.max(err / (4e-3 * bound + 1e-5))) <= 1.5
+
+
+@pytest.mark.parametrize("M,K,N,parts", [(1, 4096, 1096, 3), (16, 2048, 4096, 4), (5, 1024, 200, 2)])
+def test_column_shards_reassemble_to_the_full_product(M, K, N, parts):
+    """Section 4.4: every worker owns distinct output columns and needs nothing from the others.  Each shard's GEMV
+    (blob cut out by tf_pack_shard, N = the shard's column count) fills its column range of y; the assembled result
+    passes parity against the oracle on the whole matrix."""
+    p = wl.make_w4(M, K, N, seed=1600 + M)
+    full = gu.pack(p)
+    a = gu.to_device_bf16(p.a_bf16)
+    y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMV_W4A16, M, K, N), dtype=torch.uint8, device="cuda")
+    for part in range(parts):
+        n0, nc = tf.tf_shard_columns(N, part, parts)
+        shard = torch.from_numpy(tf.tf_pack_shard(full, part, parts)).cuda()
+        y_part = torch.empty((M, nc), dtype=torch.bfloat16, device="cuda")
+        tf.tf_gemv_w4a16(shard, a, y_part, M, K, nc, ws)
+        y[:, n0:n0 + nc] = y_part
+    assert tf.tf_device_status(ws) == 0
+    gu.check_against_oracle(p, gu.bits_of(y))

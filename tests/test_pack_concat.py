@@ -79,3 +79,35 @@ def test_concat_rejects_what_it_cannot_join():
     with pytest.raises(tf.TileFuseError) as e:
         tf.tf_pack_concat([bw, bw, bw])
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("bits,K,N,g,parts", [(4, 256, 200, 128, 2), (4, 384, 328, 64, 3), (8, 256, 136, 128, 3), (4, 128, 64, 32, 1)])
+def test_pack_shard_is_the_packer_on_the_column_slice(bits, K, N, g, parts):
+    """tf_pack_shard cuts a column range out of a blob: byte for byte what the packer gives for the sliced inputs,
+    and the shards tile the columns without gap or overlap."""
+    p = wl.make_w4(1, K, N, seed=77, group_size=g, keep_raw=True) if bits == 4 else wl.make_w8(1, K, N, seed=77, group_size=g)
+    full = (tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, K, N, g) if bits == 4 else tf.tf_pack_w8(p.w_i8, p.scales_f16, K, N, g))
+    covered = 0
+    for part in range(parts):
+        n0, nc = tf.tf_shard_columns(N, part, parts)
+        assert n0 == covered and nc > 0 and n0 % 64 == 0
+        covered += nc
+        shard = tf.tf_pack_shard(full, part, parts)
+        if bits == 4:
+            q, z = p.raw["q"][:, n0:n0 + nc], p.raw["z"][:, n0:n0 + nc]
+            want = tf.tf_pack_awq(wl.awq_pack_words(q), np.ascontiguousarray(p.scales_f16[:, n0:n0 + nc]), wl.awq_pack_words(z), K, nc, g)
+        else:
+            want = tf.tf_pack_w8(np.ascontiguousarray(p.w_i8[:, n0:n0 + nc]), np.ascontiguousarray(p.scales_f16[:, n0:n0 + nc]), K, nc, g)
+        assert np.array_equal(shard, want)
+    assert covered == N
+
+
+def test_pack_shard_errors():
+    p = wl.make_w4(1, 128, 64, seed=78)
+    full = tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, 128, 64)
+    L = tf.lib()
+    out = np.zeros(full.nbytes, dtype=np.uint8)
+    assert L.tf_pack_shard(full.ctypes.data, 0, 2, out.ctypes.data, out.nbytes) == 2        # more parts than strips
+    assert L.tf_pack_shard(full.ctypes.data, 1, 1, out.ctypes.data, out.nbytes) == 2        # part outside 0..parts-1
+    assert L.tf_pack_shard(full.ctypes.data, 0, 1, out.ctypes.data, out.nbytes - 1) == 5
+    assert L.tf_pack_shard(out.ctypes.data, 0, 1, full.ctypes.data, full.nbytes) == 4       # not a blob
