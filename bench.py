@@ -723,6 +723,23 @@ def run_gpu(args):
                 layout[f"{M}x{K}x{N}"] = {"pretiled_us": round(t_tiled, 2), "raw_us": round(t_raw, 2)}
             del raw, tiled
         assert tf.tf_device_status(ws) == 0
+        # the GEMM arm: the pre-tiled GEMM on the offline blob against the same GEMM with the AWQ arrays re-tiled on
+        # the fly into scratch on every call (tf_gemm_awq_raw): the difference is what the offline pre-tiling removes
+        p2 = wl.config2()
+        qw = torch.from_numpy(p2.qweight.view(np.int32)).to(dev)
+        sc = torch.from_numpy(p2.scales_f16.view(np.int16)).to(dev)
+        qz = torch.from_numpy(p2.qzeros.view(np.int32)).to(dev)
+        blob = torch.from_numpy(tf.tf_pack_awq(p2.qweight, p2.scales_f16, p2.qzeros, p2.K, p2.N)).to(dev)
+        a2 = torch.from_numpy(p2.a_bf16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+        y2 = torch.empty((p2.M, p2.N), dtype=torch.bfloat16, device=dev)
+        rws = torch.zeros(tf.tf_gemm_awq_raw_workspace_size(p2.M, p2.K, p2.N, 128), dtype=torch.uint8, device=dev)
+        with torch.cuda.stream(stream):
+            t_pre = timed(lambda: tf.tf_gemm_w4a16(blob, a2, y2, p2.M, p2.K, p2.N, rws, stream=stream), 10)
+            t_raw = timed(lambda: tf.tf_gemm_awq_raw(qw, sc, qz, a2, y2, p2.M, p2.K, p2.N, 128, rws, stream=stream), 10)
+        assert tf.tf_device_status(rws) == 0
+        layout[f"gemm_{p2.M}x{p2.K}x{p2.N}"] = {"pretiled_us": round(t_pre, 2), "raw_us": round(t_raw, 2),
+                                                "note": "raw = tf_pack_awq_device into scratch + the pre-tiled GEMM, per call"}
+        del qw, sc, qz, blob, a2, y2, rws
         ablation["layout"] = layout
 
     if rank != 0:

@@ -325,6 +325,30 @@ tf_status tf_gemv_w4a16_static_status(void* cuda_stream);
 tf_status tf_gemv_awq_raw(const uint32_t* qweight, const uint16_t* scales_fp16, const uint32_t* qzeros,
                           const void* a_bf16, void* y_bf16, int M, int K, int N, int group_size,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+/*
+ * Pre-tiling on the GPU (Section 4.2's re-tiling done at run time): the AWQ arrays in device memory -> the packed
+ * blob in device memory, byte for byte what tf_pack_awq writes (header included).  Arguments as tf_pack_awq, all
+ * pointers device, 16-byte aligned; asynchronous on `cuda_stream`.
+ * Errors: TF_ERR_NULL, TF_ERR_SHAPE, TF_ERR_WORKSPACE (out_bytes < tf_packed_size), TF_ERR_ALIGN, TF_ERR_ARCH, TF_ERR_CUDA.
+ */
+tf_status tf_pack_awq_device(const uint32_t* qweight, const uint16_t* scales_fp16, const uint32_t* qzeros,
+                             int K, int N, int group_size, void* out, size_t out_bytes, void* cuda_stream);
+
+/*
+ * GEMM arm of the layout ablation (Section 5.5): the fused W4A16 GEMM computed from the AWQ arrays as given, with no
+ * offline pre-tiling -- the arrays are re-tiled into scratch memory on every call (tf_pack_awq_device) and multiplied
+ * by the pre-tiled GEMM.  The difference to tf_gemm_w4a16 on an offline blob is the cost the offline pre-tiling of
+ * Section 4.2 removes.  Arguments as tf_gemv_awq_raw, 1 <= M <= 4096, group_size 32, 64 or a multiple of 128;
+ *   workspace   device, at least tf_gemm_awq_raw_workspace_size(M, K, N, group_size) bytes (the GEMM's workspace,
+ *               then the re-tiled blob); its first TF_WORKSPACE_ZERO_BYTES must be zero before first use and are left
+ *               zero; tf_device_status reads its status word.
+ * Results are those of tf_gemm_w4a16_grouped on the blob tf_pack_awq would write.  Two kernel launches.
+ */
+tf_status tf_gemm_awq_raw(const uint32_t* qweight, const uint16_t* scales_fp16, const uint32_t* qzeros,
+                          const void* a_bf16, void* y_bf16, int M, int K, int N, int group_size,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t tf_gemm_awq_raw_workspace_size(int M, int K, int N, int group_size);
+
 /* Scratch bytes tf_gemv_awq_raw needs on the current device (0 if the shape is illegal or the device is
  * not compute capability 10.x). */
 size_t tf_gemv_awq_raw_workspace_size(int M, int K, int N, int group_size);

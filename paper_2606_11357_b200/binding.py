@@ -24,7 +24,8 @@ EXPORTS = ("tf_packed_size", "tf_pack_awq", "tf_pack_w8", "tf_pack_concat", "tf_
            "tf_gemv_w4a16", "tf_gemv_w8a16", "tf_gemm_w4a16", "tf_gemm_w8a16",
            "tf_workspace_size", "tf_device_status", "tf_status_string", "tf_version", "tf_gemv_w4a16_static",
            "tf_dequant_bf16", "tf_gemv_awq_raw", "tf_gemv_awq_raw_workspace_size", "tf_gemv_plan", "tf_debug_inject", "tf_gemv_w4a16_static_status",
-           "tf_gemv_w4a16_grouped", "tf_gemm_w4a16_grouped", "tf_shard_columns", "tf_pack_shard")
+           "tf_gemv_w4a16_grouped", "tf_gemm_w4a16_grouped", "tf_shard_columns", "tf_pack_shard",
+           "tf_pack_awq_device", "tf_gemm_awq_raw", "tf_gemm_awq_raw_workspace_size")
 
 
 class TileFuseError(RuntimeError):
@@ -68,6 +69,11 @@ def lib() -> ctypes.CDLL:
         L.tf_gemv_awq_raw.restype = c_int
         L.tf_gemv_awq_raw.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, c_int, vp, c_size, vp]
         L.tf_gemv_awq_raw_workspace_size.restype, L.tf_gemv_awq_raw_workspace_size.argtypes = c_size, [c_int] * 4
+        L.tf_gemm_awq_raw.restype = c_int
+        L.tf_gemm_awq_raw.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, c_int, vp, c_size, vp]
+        L.tf_gemm_awq_raw_workspace_size.restype, L.tf_gemm_awq_raw_workspace_size.argtypes = c_size, [c_int] * 4
+        L.tf_pack_awq_device.restype = c_int
+        L.tf_pack_awq_device.argtypes = [vp, vp, vp, c_int, c_int, c_int, vp, c_size, vp]
         L.tf_device_status.restype, L.tf_device_status.argtypes = c_int, [vp, vp]
         L.tf_status_string.restype, L.tf_status_string.argtypes = ctypes.c_char_p, [c_int]
         L.tf_version.restype, L.tf_version.argtypes = c_int, []
@@ -197,6 +203,23 @@ def tf_gemv_awq_raw(qweight, scales_f16, qzeros, a, y, M: int, K: int, N: int, g
     int32 [K/g, N/8]); a, y as for tf_gemv_w4a16; workspace: uint8 CUDA tensor."""
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check("tf_gemv_awq_raw", lib().tf_gemv_awq_raw(_dev(qweight), _dev(scales_f16), _dev(qzeros), _dev(a), _dev(y),
+                                                    M, K, N, group_size, _dev(workspace), ws_bytes, _stream(stream)))
+
+
+def tf_pack_awq_device(qweight, scales_f16, qzeros, K: int, N: int, group_size: int, out, stream=None) -> None:
+    """The AWQ arrays (CUDA tensors) -> the packed blob (uint8 CUDA tensor of at least tf_packed_size bytes)."""
+    _check("tf_pack_awq_device", lib().tf_pack_awq_device(_dev(qweight), _dev(scales_f16), _dev(qzeros), K, N, group_size,
+                                                          _dev(out), out.numel() * out.element_size(), _stream(stream)))
+
+
+def tf_gemm_awq_raw_workspace_size(M: int, K: int, N: int, group_size: int = 128) -> int:
+    return int(lib().tf_gemm_awq_raw_workspace_size(M, K, N, group_size))
+
+
+def tf_gemm_awq_raw(qweight, scales_f16, qzeros, a, y, M: int, K: int, N: int, group_size: int, workspace, stream=None) -> None:
+    """The fused GEMM on the AWQ arrays themselves (re-tiled into the workspace on every call, then multiplied)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check("tf_gemm_awq_raw", lib().tf_gemm_awq_raw(_dev(qweight), _dev(scales_f16), _dev(qzeros), _dev(a), _dev(y),
                                                     M, K, N, group_size, _dev(workspace), ws_bytes, _stream(stream)))
 
 

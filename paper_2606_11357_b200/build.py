@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtilefuse.so")
 OBJ = os.path.join(PKG, "build")
-SOURCES = ["pack.cpp", "api.cu", "gemv.cu", "gemv_raw.cu", "gemm.cu", "unpack.cu", "static_scratch.cu"]
+SOURCES = ["pack.cpp", "api.cu", "gemv.cu", "gemv_raw.cu", "gemm.cu", "unpack.cu", "static_scratch.cu", "repack.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false",

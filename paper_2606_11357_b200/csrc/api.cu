@@ -224,6 +224,52 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_awq_raw(cons
     return TF_OK;
 }
 
+extern "C" __attribute__((visibility("default"))) tf_status tf_pack_awq_device(const uint32_t* qweight, const uint16_t* scales,
+                                                                               const uint32_t* qzeros, int K, int N, int group_size,
+                                                                               void* out, size_t out_bytes, void* stream) {
+    if (!qweight || !scales || !qzeros || !out) return TF_ERR_NULL;
+    const size_t total = tf_packed_size(4, K, N, group_size);
+    if (total == 0) return TF_ERR_SHAPE;
+    if (out_bytes < total) return TF_ERR_WORKSPACE;
+    if (!aligned16(qweight) || !aligned16(scales) || !aligned16(qzeros) || !aligned16(out)) return TF_ERR_ALIGN;
+    DeviceInfo dev;
+    tf_status st = device_info(&dev);
+    if (st != TF_OK) return st;
+    if (tf::launch_repack_awq(qweight, scales, qzeros, out, K, N, group_size, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return TF_ERR_CUDA;
+    }
+    return TF_OK;
+}
+
+// scratch of the raw-layout GEMM: the re-tiled blob (rounded up to 256 bytes), then the GEMM's own workspace
+static size_t raw_gemm_blob_bytes(int K, int N, int group_size) {
+    return (tf_packed_size(4, K, N, group_size) + 255) / 256 * 256;
+}
+
+extern "C" __attribute__((visibility("default"))) size_t tf_gemm_awq_raw_workspace_size(int M, int K, int N, int group_size) {
+    if (M < 1 || M > TF_MAX_M_GEMM || tf_packed_size(4, K, N, group_size) == 0) return 0;
+    return raw_gemm_blob_bytes(K, N, group_size) + tf::gemm_workspace_bytes(M, K, N);
+}
+
+extern "C" __attribute__((visibility("default"))) tf_status tf_gemm_awq_raw(const uint32_t* qweight, const uint16_t* scales,
+                                                                            const uint32_t* qzeros, const void* a, void* y,
+                                                                            int M, int K, int N, int group_size,
+                                                                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (!qweight || !scales || !qzeros || !a || !y) return TF_ERR_NULL;
+    if (M < 1 || M > TF_MAX_M_GEMM) return TF_ERR_SHAPE;
+    const size_t need = tf_gemm_awq_raw_workspace_size(M, K, N, group_size);
+    if (need == 0) return TF_ERR_SHAPE;
+    if (workspace == nullptr || workspace_bytes < need) return TF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return TF_ERR_ALIGN;
+    const size_t blob_bytes = raw_gemm_blob_bytes(K, N, group_size);
+    uint8_t* gemm_ws = static_cast<uint8_t*>(workspace);                 // the GEMM's workspace first: its head holds the status word
+    uint8_t* blob = gemm_ws + tf::gemm_workspace_bytes(M, K, N);
+    tf_status st = tf_pack_awq_device(qweight, scales, qzeros, K, N, group_size, blob, blob_bytes, stream);
+    if (st != TF_OK) return st;
+    return gemm(4, blob, a, y, M, K, N, gemm_ws, tf::gemm_workspace_bytes(M, K, N), stream, group_size);
+}
+
 extern "C" __attribute__((visibility("default"))) tf_status tf_device_status(const void* workspace, void* stream) {
     if (!workspace) return TF_ERR_NULL;
     uint32_t word[4] = {0, 0, 0, 0};

@@ -108,6 +108,10 @@ cudaError_t launch_gemv_raw(const RawGemvPlan& plan, const uint32_t* qweight, co
                             const uint32_t* qzeros, const void* a, void* y, int M, int K, int N, int group_size,
                             void* workspace, cudaStream_t stream);
 
+// Pre-tiling on the GPU: the AWQ arrays (device) -> the packed blob (device), byte for byte what tf_pack_awq writes.
+cudaError_t launch_repack_awq(const uint32_t* qweight, const uint16_t* scales, const uint32_t* qzeros, void* out, int K, int N,
+                              int group_size, cudaStream_t stream);
+
 // Prefill GEMM (tcgen05).  `workspace` starts with the DeviceStatus word.
 size_t gemm_workspace_bytes(int M, int K, int N);
 cudaError_t launch_gemm(int bits, const void* blob, const void* a, void* y, int M, int K, int N,

@@ -80,3 +80,44 @@ def test_raw_gemv_one_hot_activations_pick_exact_weights():
     y = run_raw(p, a_bits=a)
     want = wl.f32_to_bf16_bits(w[ks].astype(np.float32))
     assert np.array_equal(bf16_bits_to_f64(y), bf16_bits_to_f64(want))
+
+
+def _awq_on_device(p):
+    return (torch.from_numpy(p.qweight.view(np.int32)).cuda(), torch.from_numpy(p.scales_f16.view(np.int16)).cuda(),
+            torch.from_numpy(p.qzeros.view(np.int32)).cuda())
+
+
+@pytest.mark.parametrize("K,N,g", [(128, 8, 128), (384, 72, 128), (512, 200, 256), (1024, 1096, 64), (256, 136, 32), (4096, 4096, 128)])
+def test_device_packer_writes_the_host_packers_bytes(K, N, g):
+    """Pre-tiling on the GPU: byte for byte the blob tf_pack_awq writes (header, weights, scales, zeros, padding)."""
+    p = wl.make_w4(1, K, N, seed=700 + K + g, group_size=g)
+    want = tf.tf_pack_awq(p.qweight, p.scales_f16, p.qzeros, K, N, g)
+    qw, sc, qz = _awq_on_device(p)
+    guard = 256
+    buf = torch.full((guard + want.nbytes + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    tf.tf_pack_awq_device(qw, sc, qz, K, N, g, buf[guard:guard + want.nbytes])
+    torch.cuda.synchronize()
+    got = buf.cpu().numpy()
+    assert np.all(got[:guard] == 0xA5) and np.all(got[guard + want.nbytes:] == 0xA5), "write outside the blob"
+    assert np.array_equal(got[guard:guard + want.nbytes], want)
+
+
+@pytest.mark.parametrize("M,K,N,g", [(24, 512, 200, 128), (130, 1024, 328, 64), (300, 2048, 1096, 128), (64, 256, 136, 32)])
+def test_gemm_on_the_raw_awq_arrays(M, K, N, g):
+    """The GEMM arm of the layout ablation: re-tiled on the fly, then the pre-tiled GEMM; parity against the oracle and
+    bit-identical to the pre-tiled path on the offline blob."""
+    p = wl.make_w4(M, K, N, seed=800 + M, group_size=g)
+    qw, sc, qz = _awq_on_device(p)
+    a = gu.to_device_bf16(p.a_bf16)
+    y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(tf.tf_gemm_awq_raw_workspace_size(M, K, N, g), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        tf.tf_gemm_awq_raw(qw, sc, qz, a, y, M, K, N, g, ws)
+    assert tf.tf_device_status(ws) == 0
+    gu.check_against_oracle(p, gu.bits_of(y))
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    y2 = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    ws2 = torch.zeros(tf.tf_workspace_size(tf.TF_OP_GEMM_W4A16, M, K, N), dtype=torch.uint8, device="cuda")
+    tf.tf_gemm_w4a16_grouped(blob, a, y2, M, K, N, g, ws2)
+    torch.cuda.synchronize()
+    assert np.array_equal(gu.bits_of(y), gu.bits_of(y2))
