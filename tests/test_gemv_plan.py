@@ -1,0 +1,68 @@
+"""Host logic of the GEMV launcher: the launch plan (tf_gemv_plan) for a grid of shapes, without a GPU.
+
+The plan decides grid, warps, ring depth and which kernel variant runs; a wrong plan shows up on the GPU as a
+launch failure or a hang, so its invariants are pinned here for every shape class, on the SM counts the library may
+meet."""
+import itertools
+
+import pytest
+
+from paper_2606_11357_b200 import binding as tf
+from paper_2606_11357_b200 import build as tfbuild
+
+SMEM_HALF, SMEM_WHOLE = 110 * 1024, 220 * 1024
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    tfbuild.build()
+
+
+SHAPES = [(128, 8), (128, 64), (512, 200), (4096, 1024), (4096, 4096), (4096, 14336), (14336, 4096), (4096, 32768),
+          (32768, 4096), (32768, 32768), (1024, 136), (256, 32768)]
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("sm_count", [148, 132, 80, 16])
+def test_plan_invariants(bits, sm_count):
+    for (K, N), M in itertools.product(SHAPES, (1, 2, 3, 8, 9, 16)):
+        p = tf.tf_gemv_plan(bits, M, K, N, sm_count)
+        tiles = (K // 128) * (-(-N // 64))
+        assert 1 <= p["grid"] <= 256 and p["grid"] <= max(sm_count, 1) or p["cluster"] > 1
+        assert p["threads"] == 32 * (p["consumers"] + 2) and 4 <= p["consumers"] <= 12
+        assert p["stages"] >= 2
+        assert p["cluster"] in (1, 2, 4, 8)
+        assert 1 <= p["nclusters"] <= max(p["grid"], 1)                  # CTAs (or clusters) that take part
+        if M > 8:
+            assert p["full"] == 1 and p["i8"] == 0 and p["consumers"] <= 8
+        if M <= 2:
+            assert p["i8"] == 1                                          # both formats take the integer path at 1 and 2 tokens
+        else:
+            assert p["i8"] == 0 and p["full"] == 1                       # the floating-point path takes the whole SM
+        if p["cluster"] == 1 and tiles >= sm_count:
+            assert p["grid"] == sm_count                                 # one persistent CTA per SM
+
+
+def test_plan_of_the_benchmark_shapes_on_a_b200():
+    """The shapes of the decode step on 148 SMs: which variant each gets (asserted again on the GPU by the chain tests)."""
+    kind = lambda p: "cluster" if p["cluster"] > 1 else ("whole" if p["full"] else "half")
+    for (K, N) in ((4096, 4096), (4096, 1024), (4096, 14336), (14336, 4096)):
+        assert kind(tf.tf_gemv_plan(4, 1, K, N, 148)) == "half"
+        assert kind(tf.tf_gemv_plan(4, 4, K, N, 148)) == "whole"
+    # no GPU here: the cluster-occupancy query fails, so 9..16 tokens plan for global mode
+    assert kind(tf.tf_gemv_plan(4, 16, 4096, 14336, 148)) == "whole"
+    p = tf.tf_gemv_plan(4, 1, 4096, 1024, 148)
+    assert p["grid"] == 148 and p["nclusters"] == 64                     # 64 CTAs x 8 tiles take part, the grid stays one per SM
+    p = tf.tf_gemv_plan(4, 1, 4096, 4096, 148)
+    assert p["nclusters"] == 128                                         # 128 CTAs x 16 tiles: ranges line up with the strips
+
+
+def test_plan_rejects_illegal_arguments():
+    L = tf.lib()
+    import ctypes
+    out = (ctypes.c_int * 8)()
+    ptr = ctypes.cast(out, ctypes.c_void_p)
+    assert L.tf_gemv_plan(4, 1, 4096, 4096, 148, None) == 1
+    assert L.tf_gemv_plan(5, 1, 4096, 4096, 148, ptr) == 2
+    assert L.tf_gemv_plan(4, 17, 4096, 4096, 148, ptr) == 2
+    assert L.tf_gemv_plan(4, 1, 100, 4096, 148, ptr) == 2
