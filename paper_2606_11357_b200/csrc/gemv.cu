@@ -506,13 +506,44 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     for (int e = 0; e < 4; ++e) acc[w][mt][e] = 0.f;
 
             // the warp's tiles come every nconsumers-th tile of the range, whatever segment they fall into
-            for (; j < i + seg_len; j += nconsumers) {
-                const int lj = j - i, cl = lj / kR, slot = lj - cl * kR;
+            // Find a tile of this segment in the ring, wait until it has landed and fetch the metadata of its first
+            // group.  Called once per tile, in order (the ring position only moves forward).  (Calling it for the next
+            // tile already before the current tile's scales are applied, so that the wait would run under the tail of
+            // the current tile, was measured slower: 36.9 against 35.8 us over the four shapes at 4 tokens, 53.4 against
+            // 52.3 at 16.)
+            const uint8_t* nx_tile = nullptr;
+            int nx_s = 0, nx_slot = 0, nx_cl = 0;
+            uint4 nx_sc = make_uint4(0u, 0u, 0u, 0u);
+            uint32_t nx_zw = 0u;
+            auto locate_and_wait = [&](int jj) -> bool {
+                const int lj = jj - i, cl = lj / kR, slot = lj - cl * kR;
                 const int cg = chunk_base + cl;
                 s_cur += cg - cg_cur;
                 cg_cur = cg;
                 while (s_cur >= nstages) { s_cur -= nstages; ++use_cur; }
                 const int s = s_cur;
+                if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
+                    const long long t_begin = clock64();
+                    while (stage_tag[s] != (uint32_t)cg) {
+                        if (*abort_flag != 0) return false;
+                        if (wait_expired(t_begin, abort_flag)) { *abort_flag = 0x280 + s; return false; }
+                    }
+                }
+                if (!mbar_wait(full0 + 8 * s, use_cur & 1, abort_flag, 0x200 + s)) return false;
+                nx_tile = ring + (size_t)s * stage_bytes + (size_t)slot * kTileBytes;
+                nx_s = s; nx_slot = slot; nx_cl = cl;
+                if constexpr (!I8) {
+                    nx_sc = *(reinterpret_cast<const uint4*>(nx_tile + kWeightBytes) + g);
+                    if (BITS == 4) nx_zw = *(reinterpret_cast<const uint32_t*>(nx_tile + w4_zero_offset(G, 0)) + g);
+                }
+                return true;
+            };
+            for (; j < i + seg_len; j += nconsumers) {
+                if (!locate_and_wait(j)) { aborted = true; break; }
+                const uint8_t* tile = nx_tile;
+                const int s = nx_s, slot = nx_slot, cl = nx_cl;
+                const uint4 sc_first = nx_sc;
+                const uint32_t zw_first = nx_zw;
                 const bool has_next = kAhead && j + nconsumers < ntiles;
                 int T_nx = T_act + nconsumers;                  // the warp's next tile is nconsumers tiles further along K
                 while (T_nx >= ktiles) T_nx -= ktiles;
@@ -529,17 +560,6 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     __syncwarp();                                // every lane's copies are visible to the warp
                     abuf_cur ^= 1;
                 }
-                if (stage_tag[s] != (uint32_t)cg) {            // the producer has not reached this chunk yet
-                    const long long t_begin = clock64();
-                    while (stage_tag[s] != (uint32_t)cg && !aborted) {
-                        if (*abort_flag != 0) aborted = true;
-                        else if (wait_expired(t_begin, abort_flag)) { *abort_flag = 0x280 + s; aborted = true; }
-                    }
-                    if (aborted) break;
-                }
-                if (!mbar_wait(full0 + 8 * s, use_cur & 1, abort_flag, 0x200 + s)) { aborted = true; break; }
-                const uint8_t* stage = ring + (size_t)s * stage_bytes;
-                const uint8_t* tile = stage + (size_t)slot * kTileBytes;
 
                 if constexpr (I8) {
                     const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes) + g);
@@ -684,12 +704,14 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 // ---- floating-point path: group after group (one group per tile unless the group size is 64 or 32) ----
 #pragma unroll
                 for (int gr = 0; gr < G; ++gr) {
-                    const uint4 sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes + gr * kScaleBytes) + g);
-                    uint32_t zg[4], zg8[4];
-                    if (BITS == 4) {
-                        const uint32_t zword = *(reinterpret_cast<const uint32_t*>(tile + w4_zero_offset(G, gr)) + g);
-                        w4_zero_regs(zword, zg, zg8);
+                    uint4 sc = sc_first;
+                    uint32_t zword = zw_first;
+                    if (gr > 0) {
+                        sc = *(reinterpret_cast<const uint4*>(tile + kWeightBytes + gr * kScaleBytes) + g);
+                        if (BITS == 4) zword = *(reinterpret_cast<const uint32_t*>(tile + w4_zero_offset(G, gr)) + g);
                     }
+                    uint32_t zg[4], zg8[4];
+                    if (BITS == 4) w4_zero_regs(zword, zg, zg8);
                     float gacc[4][MT][4];
 #pragma unroll
                     for (int w = 0; w < 4; ++w)
@@ -739,6 +761,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                             const int tiles_here = min(kR, seg_len - cl * kR);
                             mbar_arrive_n(empty0 + 8 * s, slot == tiles_here - 1 ? (uint32_t)(kR - tiles_here + 1) : 1u);
                         }
+
                     }
 
                     // the group's scales, in fp32 (Eq. 1 / Eq. 2 factored per group)
@@ -756,6 +779,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                         }
                     }
                 }
+                if (aborted) break;
                 }
             }
             if (aborted) break;
