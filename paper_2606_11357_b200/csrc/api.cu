@@ -137,7 +137,7 @@ extern "C" __attribute__((visibility("default"))) tf_status tf_gemv_plan(int bit
     if (sm_count > tf::kGemvMaxGrid) sm_count = tf::kGemvMaxGrid;
     const tf::GemvPlan p = tf::plan_gemv(bits, M, K, N, sm_count);
     out[0] = p.grid; out[1] = p.threads; out[2] = p.consumers; out[3] = p.stages;
-    out[4] = p.full ? 1 : 0; out[5] = p.i8 ? 1 : 0; out[6] = p.cluster; out[7] = p.nclusters;
+    out[4] = p.full ? 1 : 0; out[5] = p.i8 ? (p.piece_tab > 0 ? 2 : 1) : 0; out[6] = p.cluster; out[7] = p.nclusters;
     return TF_OK;
 }
 

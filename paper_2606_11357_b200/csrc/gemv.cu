@@ -220,11 +220,101 @@ __device__ __noinline__ bool gather_rows(float4* slot, int count, int M, float4 
 
 }  // namespace
 
+// Integer path, piece table: the activation pieces of the k-tiles of a CTA's range, prepared once.  Entry e holds
+// k-tile (t_first + e) mod ktiles: per token three piece columns of 32 words (the word of k-block kb and k quarter t at
+// t * 8 + kb, so that a thread of the MMA phase finds the eight k-blocks of its column and quarter in two 16-byte
+// loads), then 8 column entries {2^(emax-148) 256^j, sum of the piece over the tile}.  kLanes lanes prepare one
+// entry (lane u of the group holds kVals consecutive k), a warp 32 / kLanes entries per pass.  Not inlined: the
+// table is filled once per kernel, and inlined it took registers from the tile loop (spills that were reloaded per
+// tile: a whole-SM range of 111 tiles ran 0.5 us longer).
+template <int BITS, int kLanes>
+__device__ __noinline__ void fill_piece_table(uint32_t* pscr, const __nv_bfloat16* __restrict__ a_glob, int M, int K, int ktiles,
+                                              int T_first, int piece_n, int cw, int nconsumers, int lane) {
+    constexpr int kVals = 128 / kLanes, kPerPass = 32 / kLanes, kColWords = 32;
+    const int piece_entry_words = (kGemvPieceEntryBytes / 4) * M;
+    const int b = lane / kLanes, u = lane % kLanes;
+    for (int e0 = kPerPass * cw; e0 < piece_n; e0 += kPerPass * nconsumers) {
+        const int e = e0 + b;
+        const bool live = e < piece_n;
+        int T = T_first + e;                    // e < ktiles
+        if (T >= ktiles) T -= ktiles;
+        uint32_t* ent = pscr + (size_t)(live ? e : 0) * piece_entry_words;
+        uint2* meta = reinterpret_cast<uint2*>(ent + 96 * M);
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            if (m < M) {
+                uint32_t x[kVals / 2];
+                const __nv_bfloat16* src = a_glob + (size_t)m * K + (size_t)T * kTileK + kVals * u;
+                if constexpr (kVals == 4) {
+                    uint2 r = make_uint2(0u, 0u);
+                    if (live) r = __ldcg(reinterpret_cast<const uint2*>(src));
+                    x[0] = r.x; x[1] = r.y;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kVals / 8; ++i) {
+                        uint4 r = make_uint4(0u, 0u, 0u, 0u);
+                        if (live) r = __ldcg(reinterpret_cast<const uint4*>(src) + i);
+                        x[4 * i] = r.x; x[4 * i + 1] = r.y; x[4 * i + 2] = r.z; x[4 * i + 3] = r.w;
+                    }
+                }
+                uint32_t ex = 0u;
+#pragma unroll
+                for (int i = 0; i < kVals / 2; ++i) ex = max(ex, max((x[i] << 17) >> 24, (x[i] << 1) >> 24));
+#pragma unroll
+                for (int d = 1; d < kLanes; d *= 2) ex = max(ex, __shfl_xor_sync(0xFFFFFFFFu, ex, d));
+                ex = max(ex, 22u);                                    // keeps both powers of two normal numbers
+                const float mult = __uint_as_float((275u - ex) << 23);                // 2^(148 - emax)
+                // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
+                const float se = ex == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((ex - 21u) << 23);
+                int psum[3] = {0, 0, 0};
+#pragma unroll
+                for (int q = 0; q < kVals / 4; ++q) {           // four consecutive k: one word per piece
+                    const int k0 = kVals * u + 4 * q;           // k-block k0 / 16, k quarter (k0 % 16) / 4
+                    const uint32_t x0 = x[2 * q], x1 = x[2 * q + 1];
+                    uint32_t v[4];
+                    v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
+                    v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
+                    v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
+                    v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
+                    const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
+                    const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
+                    uint32_t word[3];
+                    word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+                    word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
+                    word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {
+                        if (live) ent[(3 * m + j) * kColWords + ((k0 >> 2) & 3) * 8 + (k0 >> 4)] = word[j];
+                        if constexpr (BITS == 4) psum[j] = __dp4a((int)word[j], 0x01010101, psum[j]);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 3; ++j) {
+                    if constexpr (BITS == 4) {                  // sum of the piece over the tile's 128 k, for the zero point
+#pragma unroll
+                        for (int d = 1; d < kLanes; d *= 2) psum[j] += __shfl_xor_sync(0xFFFFFFFFu, psum[j], d);
+                    }
+                    if (live && u == 0)
+                        meta[3 * m + j] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum[j]);
+                }
+            }
+        }
+        if (live && u == 0) {                           // columns without a token contribute nothing
+#pragma unroll
+            for (int c = 3; c < 8; ++c)
+                if (c >= 3 * M) meta[c] = make_uint2(0u, 0u);
+        }
+    }
+}
+
 // G = groups per tile: 1 for group sizes that are multiples of 128, 2 / 4 for the 4-bit group sizes 64 / 32.
-template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
-__global__ void __launch_bounds__(gemv_max_threads(MT, FULL), FULL ? 1 : 2)
+// I8 = 0: floating-point path; 1: integer path, every consumer warp prepares the activation pieces of the tile it
+// works on; 2: integer path, the consumer warps prepare the pieces of every k-tile of the CTA's range once, before
+// the first tile, into a table all of them read (ranges that pass over the same k-tiles several times).
+template <int BITS, int MT, bool FULL, bool CL, int I8, int G = 1>
+__global__ void __launch_bounds__(gemv_max_threads(MT, FULL, I8 != 0), FULL ? 1 : 2)
 gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
-                   int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes, int nred,
+                   int nstages, int stage_bytes, int csize, int nclusters, int xslot_bytes, int nred, int piece_tab,
                    uint8_t* __restrict__ workspace, uint32_t debug) {
     static_assert(G == 1 || (BITS == 4 && !I8 && !CL && FULL), "several groups per tile: 4-bit, floating-point path, whole SM");
     constexpr int kTileBytes = tile_bytes(BITS, G);
@@ -247,10 +337,11 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     float* red = reinterpret_cast<float*>(smem + kGemvBarrierBytes);
     // xred [csize][xslot]: in cluster mode, the partials other CTAs of the cluster send to the finisher of a strip
     uint8_t* xred = smem + kGemvBarrierBytes + nred * nconsumers * kRedWarp * 4;
-    // pscr [consumers][1 KB]: integer path, a warp's activation pieces of the tile it works on
+    // pscr: integer path.  [consumers][1 KB], a warp's activation pieces of the tile it works on; or
+    // [piece_tab][kGemvPieceEntryBytes per token], the pieces of every k-tile of the CTA's range
     uint32_t* pscr = reinterpret_cast<uint32_t*>(xred + ((CL && csize > 1 ? csize * xslot_bytes : 0) + 1023) / 1024 * 1024);
     // abuf [consumers][2][16 rows of kActRowBytes]: 9..16 tokens, a warp's activations of the tile it works on and of its next one
-    uint8_t* abuf = reinterpret_cast<uint8_t*>(pscr) + (I8 ? nconsumers * 1024 : 0);
+    uint8_t* abuf = reinterpret_cast<uint8_t*>(pscr) + (I8 == 2 ? (piece_tab * kGemvPieceEntryBytes * M + 1023) / 1024 * 1024 : I8 == 1 ? nconsumers * 1024 : 0);
     uint8_t* ring = abuf + (MT == 2 ? nconsumers * kGemvActWarpBytes : 0);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -451,7 +542,70 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         auto load_ag_kb = [&](const __nv_bfloat16* base, int kb) {
             if (g < M) ag[0][kRegActs ? kb : 0] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)g * K + 4 * t + 16 * kb));
         };
+        // Integer path: the activation pieces of one (k-tile, token) pair, from the raw bf16 of lane L (k = 4L .. 4L+3).
+        // dst: [column][kColWords] piece words, the word of lane L at (L & 3) * 8 + (L >> 2), so that a thread of the
+        // MMA phase finds the eight k-blocks of its column and k quarter in two 16-byte loads; meta: [column]
+        // {2^(emax-148) 256^j, sum of the piece over the tile} in 8-byte entries, a thread's two columns = one 16-byte
+        // load (with 4-byte entries and an 8-byte load the same kernel ran 12 % slower: measured, cause not established).
+        constexpr int kColWords = I8 == 2 ? 32 : 36;
+        auto make_pieces = [&](const uint2 (&raws)[2], uint32_t* dst, uint2* meta) {
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                if (m < M) {
+                    const uint2 raw = raws[m];
+                    const uint32_t x0 = raw.x, x1 = raw.y;
+                    uint32_t e = max(max((x0 << 17) >> 24, (x0 << 1) >> 24), max((x1 << 17) >> 24, (x1 << 1) >> 24));
+                    e = __reduce_max_sync(0xFFFFFFFFu, e);
+                    e = max(e, 22u);                                  // keeps both powers of two normal numbers
+                    const float mult = __uint_as_float((275u - e) << 23);          // 2^(148 - emax)
+                    // v + 0x808080 has the bytes p0 + 128, p1 + 128, p2 + 128 of the balanced split
+                    uint32_t v[4];
+                    v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
+                    v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
+                    v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
+                    v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
+                    // 4 x 3 byte transpose: one word per piece, bytes in the k order of the weight operand's bytes
+                    // (int8: k, k+1, k+2, k+3; 4-bit: k, k+2, k+1, k+3, the order of a packed word's nibble pairs)
+                    const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
+                    const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
+                    uint32_t word[3];
+                    word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+                    word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
+                    word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+                    // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
+                    const float se = e == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((e - 21u) << 23);
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {
+                        const int c = 3 * m + j;
+                        dst[c * kColWords + (lane & 3) * 8 + (lane >> 2)] = word[j];
+                        int psum = 0;                           // 4-bit: sum of the piece over the tile's 128 k, for the zero point
+                        if constexpr (BITS == 4) psum = __reduce_add_sync(0xFFFFFFFFu, __dp4a((int)word[j], 0x01010101, 0));
+                        if (lane == 0) meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum);
+                    }
+                }
+            }
+            if (lane == 0) {                                    // columns without a token contribute nothing
+#pragma unroll
+                for (int c = 3; c < 8; ++c)
+                    if (c >= 3 * M) meta[c] = make_uint2(0u, 0u);
+            }
+        };
         grid_dependency_wait();                         // the activations belong to earlier kernels until now
+        // Piece table: entry e holds k-tile (t0 + e) mod ktiles, so local tile j of the range finds its pieces in
+        // entry j mod piece_n, piece_n = min(ntiles, ktiles).  kLanes lanes prepare one entry (lane u of the group holds
+        // kVals consecutive k), a warp 32 / kLanes entries per pass, so that the 32 k-tiles of K = 4096 are one pass of
+        // all consumer warps (8 warps x 4 entries in the half-SM form, 16 x 2 in the whole-SM form); then the consumer
+        // warps meet.  (One entry per warp and pass, four passes one after the other, took about 1 us in the half-SM
+        // form: more than the table saved on a range of 48 tiles.)
+        const int piece_entry_words = (kGemvPieceEntryBytes / 4) * M;
+        const int piece_n = min(ntiles, ktiles);
+        const int T_first = t0 % ktiles;                // k-tile index of the range's first tile
+        int piece_e = 0;
+        if constexpr (I8 == 2) {
+            fill_piece_table<BITS, FULL ? 16 : 8>(pscr, a_glob, M, K, ktiles, T_first, piece_n, cw, nconsumers, lane);
+            asm volatile("bar.sync 1, %0;" ::"r"(nconsumers * 32) : "memory");
+            if (piece_n > 0) piece_e = cw % piece_n;
+        }
         if constexpr (kRegActs) {
 #pragma unroll
             for (int kb = 0; kb < 8; ++kb) ag[0][kb] = make_uint2(0u, 0u);
@@ -485,13 +639,13 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         int abuf_cur = 0;
         if (kAhead && cw < ntiles) {
             const __nv_bfloat16* base = a_glob + (size_t)T_act * kTileK;
-            if constexpr (I8) load_araw(base);
-            else {
+            if constexpr (I8 == 1) load_araw(base);
+            else if constexpr (I8 == 0) {
 #pragma unroll
                 for (int kb = 0; kb < 8; ++kb) load_ag_kb(base, kb);
             }
         }
-        int T0 = t0 % ktiles;                           // k-tile index at which the current segment starts (0 after the first)
+        int T0 = T_first;                               // k-tile index at which the current segment starts (0 after the first)
         int j = cw;                                     // this warp's next tile, as a local index of the CTA's range
         while (i < ntiles && !aborted) {
             const int seg_len = min(ntiles - i, ktiles - T0);
@@ -575,65 +729,33 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     //     4-bit: D[n][3m+j] -= z[n] sum_k p_j[m][k]       (the zero point of Eq. 2, still exact)
                     //     y[m][n] += s[n] 2^(emax-148) sum_j 256^j D[n][3m+j]
                     static_assert(!I8 || MT == 1, "the integer path is built for up to 2 tokens");
-                    uint32_t* scr = pscr + cw * 256;                    // [column][36 words]: word of lane L at (L&3)*8 + (L>>2)
-                    // [column]: 2^(emax-148) 256^j in 8-byte entries behind the 6 x 36 words, a thread's two columns = one 16-byte load
-                    // (with 4-byte entries and an 8-byte load the same kernel ran 12 % slower: measured, cause not established)
-                    uint2* col_meta = reinterpret_cast<uint2*>(scr + 216);
-#pragma unroll
-                    for (int m = 0; m < 2; ++m) {
-                        if (m < M) {
-                            // lane L holds k = 4L .. 4L+3 of the tile
-                            const uint2 raw = araw[m];
-                            const uint32_t x0 = raw.x, x1 = raw.y;
-                            uint32_t e = max(max((x0 << 17) >> 24, (x0 << 1) >> 24), max((x1 << 17) >> 24, (x1 << 1) >> 24));
-                            e = __reduce_max_sync(0xFFFFFFFFu, e);
-                            e = max(e, 22u);                                  // keeps both powers of two normal numbers
-                            const float mult = __uint_as_float((275u - e) << 23);          // 2^(148 - emax)
-                            // v + 0x808080 has the bytes p0 + 128, p1 + 128, p2 + 128 of the balanced split
-                            uint32_t v[4];
-                            v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
-                            v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
-                            v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
-                            v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
-                            // 4 x 3 byte transpose: one word per piece, bytes in the k order of the weight operand's bytes
-                            // (int8: k, k+1, k+2, k+3; 4-bit: k, k+2, k+1, k+3, the order of a packed word's nibble pairs)
-                            const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
-                            const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
-                            uint32_t word[3];
-                            word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
-                            word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
-                            word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
-                            // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
-                            const float se = e == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((e - 21u) << 23);
-#pragma unroll
-                            for (int j = 0; j < 3; ++j) {
-                                const int c = 3 * m + j;
-                                scr[c * 36 + (lane & 3) * 8 + (lane >> 2)] = word[j];
-                                int psum = 0;                           // 4-bit: sum of the piece over the tile's 128 k, for the zero point
-                                if constexpr (BITS == 4) psum = __reduce_add_sync(0xFFFFFFFFu, __dp4a((int)word[j], 0x01010101, 0));
-                                if (lane == 0) col_meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum);
-                            }
-                        }
+                    const uint32_t* scr;                                // this tile's piece words and column metadata
+                    const uint2* col_meta;
+                    if constexpr (I8 == 2) {
+                        scr = pscr + piece_e * piece_entry_words;
+                        col_meta = reinterpret_cast<const uint2*>(scr + 96 * M);
+                        piece_e += nconsumers;                          // the warp's next tile is nconsumers k-tiles further
+                        while (piece_e >= piece_n) piece_e -= piece_n;
+                    } else {
+                        uint32_t* mine_scr = pscr + cw * 256;
+                        make_pieces(araw, mine_scr, reinterpret_cast<uint2*>(mine_scr + 216));
+                        scr = mine_scr;
+                        col_meta = reinterpret_cast<const uint2*>(mine_scr + 216);
+                        if (has_next) load_araw(next_base);             // the next tile's activations, under this tile's MMAs
+                        __syncwarp();
                     }
-                    if (has_next) load_araw(next_base);                 // the next tile's activations, under this tile's MMAs
-                    if (lane == 0) {                                    // columns without a token contribute nothing
-#pragma unroll
-                        for (int c = 3; c < 8; ++c)
-                            if (c >= 3 * M) col_meta[c] = make_uint2(0u, 0u);
-                    }
-                    __syncwarp();
                     const uint4 cm = *reinterpret_cast<const uint4*>(col_meta + 2 * t);
                     const float2 col_scale = make_float2(__uint_as_float(cm.x), __uint_as_float(cm.z));
                     uint32_t bw[8];                                     // column g: the words of k-blocks 0..7 for this t
 #pragma unroll
                     for (int i = 0; i < 8; ++i) bw[i] = 0u;
                     if (g < 3 * M) {
-                        const uint4 lo = *reinterpret_cast<const uint4*>(scr + g * 36 + t * 8);
-                        const uint4 hi = *reinterpret_cast<const uint4*>(scr + g * 36 + t * 8 + 4);
+                        const uint4 lo = *reinterpret_cast<const uint4*>(scr + g * kColWords + t * 8);
+                        const uint4 hi = *reinterpret_cast<const uint4*>(scr + g * kColWords + t * 8 + 4);
                         bw[0] = lo.x; bw[1] = lo.y; bw[2] = lo.z; bw[3] = lo.w;
                         bw[4] = hi.x; bw[5] = hi.y; bw[6] = hi.z; bw[7] = hi.w;
                     }
-                    __syncwarp();                                       // the scratch is rewritten for the next tile
+                    if constexpr (I8 == 1) __syncwarp();                // the scratch is rewritten for the next tile
                     int d[4][4];
                     if constexpr (BITS == 4) {
 #pragma unroll
@@ -987,11 +1109,12 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // gain more from the next GEMV's CTAs sitting beside this one's with their rings already full, long ones
     // amortise the start of the kernel and take the whole SM too.
     const bool i8_path = M <= kGemvI8MaxM && groups == 1;     // several groups per tile: floating-point path only
-    p.full = mt == 2 || !i8_path || tiles_per_cta * tile_bytes(bits, groups) >= kGemvFullFromBytesI8;
+    p.full = mt == 2 || !i8_path || tiles_per_cta * tile_bytes(bits, groups) >= (bits == 8 ? kGemvFullFromBytesI8W8 : kGemvFullFromBytesI8W4);
     p.i8 = i8_path && p.cluster == 1;
-    // the integer path leaves the warps waiting for data, not for issue slots: 8 of them keep more tiles in flight
-    // (4096x14336, 1 token: 13.7 us with 8 warps, 14.2 us with 12)
-    p.consumers = p.i8 && p.full ? 8 : gemv_max_consumers(mt, p.full);
+    // whole-SM integer path: about 66 KB of tiles in the consumer warps' hands (16 warps on 4-bit tiles, 8 on int8 tiles)
+    // and the rest of the ring in flight.  Measured alone, one token: 4096x32768 4-bit 20.7 us half SM, 20.7 / 18.8 /
+    // 18.1 whole SM with 8 / 12 / 16 warps; 4096x14336 int8 15.8 us half SM, 12.7 / 13.3 / 14.6 whole SM with 8 / 12 / 16.
+    p.consumers = p.i8 && p.full ? gemv_i8_full_consumers(bits) : gemv_max_consumers(mt, p.full);
     if (tiles_per_cta < p.consumers) p.consumers = tiles_per_cta < 4 ? 4 : tiles_per_cta;
     p.threads = 32 * (p.consumers + 2);          // + producer warp + reducer warp
     const int kr = gemv_chunk_tiles(bits);
@@ -1002,14 +1125,28 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // two buffers for the consumer warps' partial sums where the whole SM is taken (a boundary between strips then
     // costs a fast warp nothing; measured below), one in the half-SM form, where the second would cost a ring stage
     p.nred = p.full ? 2 : 1;
-    const int fixed = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.nred * p.consumers * 8 * mt * kTileN * 4 +
-                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (p.i8 ? p.consumers * 1024 : 0) +
-                      (mt == 2 ? p.consumers * kGemvActWarpBytes : 0);
+    const int base = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.nred * p.consumers * 8 * mt * kTileN * 4 +
+                     (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (mt == 2 ? p.consumers * kGemvActWarpBytes : 0);
+    int fixed = base + (p.i8 ? p.consumers * 1024 : 0);
     int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
     if (stages > kGemvMaxStages) stages = kGemvMaxStages;
     // no more stages than the range has chunks
     const int chunks = (tiles_per_cta + kr - 1) / kr + 2;
     if (stages > chunks) stages = chunks;
+    // Integer path: a range that passes over the same k-tiles several times prepares the activation pieces of each
+    // k-tile once per CTA instead of once per tile, if the table costs the ring no stage.
+    p.piece_tab = 0;
+    if (p.i8) {
+        const int entries = tiles_per_cta < p.ktiles ? tiles_per_cta : p.ktiles;
+        const int table = (entries * kGemvPieceEntryBytes * M + 1023) / 1024 * 1024;
+        int with = (gemv_smem_budget(mt, p.full) - (base + table)) / p.stage_bytes;
+        if (with > kGemvMaxStages) with = kGemvMaxStages;
+        if (with > chunks) with = chunks;
+        if (with >= stages && tiles_per_cta * 100 >= p.ktiles * TF_PIECE_TAB_MIN_REUSE_PCT) {
+            p.piece_tab = entries;
+            fixed = base + table;
+        }
+    }
     p.stages = stages;
     p.smem_bytes = fixed + p.stages * p.stage_bytes;
     return p;
@@ -1047,7 +1184,7 @@ void note_whole_sm_launch(cudaStream_t stream) { note_launch(stream, true); }
 
 // Function attributes belong to one device: set once per device and kernel instantiation.  The flag is atomic: two
 // host threads may both find it unset and both set the attributes, which is harmless.
-template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
+template <int BITS, int MT, bool FULL, bool CL, int I8, int G = 1>
 static cudaError_t configure_one() {
     static std::atomic<bool> configured_on[kGemvMaxDevices];
     int dev = 0;
@@ -1071,14 +1208,15 @@ template <int BITS>
 static cudaError_t configure_bits() {
     cudaError_t e = cudaSuccess;
     auto all = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
-    all(configure_one<BITS, 1, false, false, false>()); all(configure_one<BITS, 1, true, false, false>());
-    all(configure_one<BITS, 1, false, false, true>());  all(configure_one<BITS, 1, true, false, true>());
-    all(configure_one<BITS, 2, true, false, false>());
-    all(configure_one<BITS, 1, false, true, false>());  all(configure_one<BITS, 1, true, true, false>());
-    all(configure_one<BITS, 2, true, true, false>());
+    all(configure_one<BITS, 1, false, false, 0>()); all(configure_one<BITS, 1, true, false, 0>());
+    all(configure_one<BITS, 1, false, false, 1>());  all(configure_one<BITS, 1, true, false, 1>());
+    all(configure_one<BITS, 1, false, false, 2>());  all(configure_one<BITS, 1, true, false, 2>());
+    all(configure_one<BITS, 2, true, false, 0>());
+    all(configure_one<BITS, 1, false, true, 0>());  all(configure_one<BITS, 1, true, true, 0>());
+    all(configure_one<BITS, 2, true, true, 0>());
     if constexpr (BITS == 4) {
-        all(configure_one<4, 1, true, false, false, 2>()); all(configure_one<4, 2, true, false, false, 2>());
-        all(configure_one<4, 1, true, false, false, 4>()); all(configure_one<4, 2, true, false, false, 4>());
+        all(configure_one<4, 1, true, false, 0, 2>()); all(configure_one<4, 2, true, false, 0, 2>());
+        all(configure_one<4, 1, true, false, 0, 4>()); all(configure_one<4, 2, true, false, 0, 4>());
     }
     return e;
 }
@@ -1092,7 +1230,7 @@ cudaError_t configure_gemv_kernels() {
     return e;
 }
 
-template <int BITS, int MT, bool FULL, bool CL, bool I8, int G = 1>
+template <int BITS, int MT, bool FULL, bool CL, int I8, int G = 1>
 static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,
                               int N, void* workspace, cudaStream_t stream) {
     cudaError_t ce = configure_one<BITS, MT, FULL, CL, I8, G>();
@@ -1126,7 +1264,7 @@ static cudaError_t launch_one(const GemvPlan& p, const void* blob, const void* a
     }
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<BITS, MT, FULL, CL, I8, G>, static_cast<const uint8_t*>(blob),
                               static_cast<const __nv_bfloat16*>(a), static_cast<__nv_bfloat16*>(y), M, K, N, p.ktiles, p.total_tiles, p.stages, p.stage_bytes,
-                              p.cluster, p.nclusters, p.xslot_bytes, p.nred, static_cast<uint8_t*>(workspace), debug_word());
+                              p.cluster, p.nclusters, p.xslot_bytes, p.nred, p.piece_tab, static_cast<uint8_t*>(workspace), debug_word());
 }
 
 template <int BITS>
@@ -1135,25 +1273,28 @@ static cudaError_t launch_bits(const GemvPlan& p, const void* blob, const void* 
     if constexpr (BITS == 4) {
         // group sizes 64 and 32: the whole-SM floating-point kernel with two or four groups per tile
         if (p.groups == 2)
-            return M > 8 ? launch_one<4, 2, true, false, false, 2>(p, blob, a, y, M, K, N, workspace, stream)
-                         : launch_one<4, 1, true, false, false, 2>(p, blob, a, y, M, K, N, workspace, stream);
+            return M > 8 ? launch_one<4, 2, true, false, 0, 2>(p, blob, a, y, M, K, N, workspace, stream)
+                         : launch_one<4, 1, true, false, 0, 2>(p, blob, a, y, M, K, N, workspace, stream);
         if (p.groups == 4)
-            return M > 8 ? launch_one<4, 2, true, false, false, 4>(p, blob, a, y, M, K, N, workspace, stream)
-                         : launch_one<4, 1, true, false, false, 4>(p, blob, a, y, M, K, N, workspace, stream);
+            return M > 8 ? launch_one<4, 2, true, false, 0, 4>(p, blob, a, y, M, K, N, workspace, stream)
+                         : launch_one<4, 1, true, false, 0, 4>(p, blob, a, y, M, K, N, workspace, stream);
     }
     if (p.groups != 1) return cudaErrorInvalidValue;
     // the cluster instructions are compiled only into the instantiations that are launched as clusters
     if (p.cluster > 1) {
-        if (M > 8) return launch_one<BITS, 2, true, true, false>(p, blob, a, y, M, K, N, workspace, stream);
-        return p.full ? launch_one<BITS, 1, true, true, false>(p, blob, a, y, M, K, N, workspace, stream)
-                      : launch_one<BITS, 1, false, true, false>(p, blob, a, y, M, K, N, workspace, stream);
+        if (M > 8) return launch_one<BITS, 2, true, true, 0>(p, blob, a, y, M, K, N, workspace, stream);
+        return p.full ? launch_one<BITS, 1, true, true, 0>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<BITS, 1, false, true, 0>(p, blob, a, y, M, K, N, workspace, stream);
     }
-    if (M > 8) return launch_one<BITS, 2, true, false, false>(p, blob, a, y, M, K, N, workspace, stream);
+    if (M > 8) return launch_one<BITS, 2, true, false, 0>(p, blob, a, y, M, K, N, workspace, stream);
+    if (p.i8 && p.piece_tab > 0)
+        return p.full ? launch_one<BITS, 1, true, false, 2>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<BITS, 1, false, false, 2>(p, blob, a, y, M, K, N, workspace, stream);
     if (p.i8)
-        return p.full ? launch_one<BITS, 1, true, false, true>(p, blob, a, y, M, K, N, workspace, stream)
-                      : launch_one<BITS, 1, false, false, true>(p, blob, a, y, M, K, N, workspace, stream);
-    return p.full ? launch_one<BITS, 1, true, false, false>(p, blob, a, y, M, K, N, workspace, stream)
-                  : launch_one<BITS, 1, false, false, false>(p, blob, a, y, M, K, N, workspace, stream);
+        return p.full ? launch_one<BITS, 1, true, false, 1>(p, blob, a, y, M, K, N, workspace, stream)
+                      : launch_one<BITS, 1, false, false, 1>(p, blob, a, y, M, K, N, workspace, stream);
+    return p.full ? launch_one<BITS, 1, true, false, 0>(p, blob, a, y, M, K, N, workspace, stream)
+                  : launch_one<BITS, 1, false, false, 0>(p, blob, a, y, M, K, N, workspace, stream);
 }
 
 cudaError_t launch_gemv(int bits, const GemvPlan& p, const void* blob, const void* a, void* y, int M, int K,

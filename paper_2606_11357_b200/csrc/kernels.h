@@ -5,12 +5,23 @@
 
 namespace tf {
 
+// Tuning knobs of the integer path (overridable at compile time for measurements).
+#ifndef TF_I8_FULL_BYTES_W4
+#define TF_I8_FULL_BYTES_W4 (288 * 1024)
+#endif
+#ifndef TF_I8_FULL_BYTES_W8
+#define TF_I8_FULL_BYTES_W8 (160 * 1024)
+#endif
+
 // ---- GEMV (persistent streaming kernel) ----------------------------------------------------------
-// Three configurations, chosen by plan_gemv:
+// Configurations, chosen by plan_gemv:
 //   integer path (1 and 2 tokens), short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs
 //     fit beside this one's and have their rings full of weights when this kernel completes.
-//   floating-point path up to 8 tokens, and long integer-path ranges: the whole SM, 12 consumer warps (8 on the
-//     integer path) and a ring deep enough to keep HBM busy while 12 tiles are being consumed.  A consumer warp
+//   integer path, long ranges: the whole SM, a ring of seven to ten stages, and as many consumer warps as hold
+//     about 66 KB of tiles (16 on 4-bit tiles, 8 on int8 tiles); where the range passes over the same k-tiles at
+//     least twice the activation pieces are prepared once per CTA (piece table) instead of once per tile.
+//   floating-point path up to 8 tokens: the whole SM, 12 consumer warps and a ring deep enough to keep HBM busy
+//     while 12 tiles are being consumed.  A consumer warp
 //     of the floating-point path is bound by instruction issue (about 20 issue cycles per packed word of 8
 //     weights, measured on registers alone), and since a GEMV may not read its activations before the kernel ahead
 //     of it has completed, only one kernel's consumers work on an SM at a time: three warps per scheduler beat two
@@ -19,15 +30,30 @@ namespace tf {
 //     warp is working on is a tile that is not in flight (measured on the four layer shapes with the ring holding
 //     weights only: 8 warps 7.9 / 4.1 / 14.5 / 15.4 us, 10 warps 8.4 / 4.1 / 15.2 / 16.1 us; 12 warps do not fit the
 //     register file).
-__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full) { return mt == 1 ? (full ? 12 : 8) : 8; }
-__host__ __device__ constexpr int gemv_max_threads(int mt, bool full) { return 32 * (gemv_max_consumers(mt, full) + 2); }   // + producer + reducer
+__host__ __device__ constexpr int gemv_max_consumers(int mt, bool full, bool i8 = false) { return mt == 1 ? (full ? (i8 ? 16 : 12) : 8) : 8; }
+__host__ __device__ constexpr int gemv_max_threads(int mt, bool full, bool i8 = false) { return 32 * (gemv_max_consumers(mt, full, i8) + 2); }   // + producer + reducer
 __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (mt == 1 && !full ? 110 : 220) * 1024; }
 // Shared memory a half-SM CTA asks for when two of its kind must not share an SM: with 228 KB per SM and 1 KB reserved
 // per CTA, two of these do not fit (2 x 115 KB), one beside a plain half-SM CTA (at most 110 KB) does.
 constexpr int kGemvSoloSmemBytes = 114 * 1024;
-// Packed bytes per CTA from which the integer path uses the whole-SM configuration (8 consumer warps in both forms;
-// measured on int8 weights: 562 KB per CTA 16.6 us half, 17.7 whole; 787 KB: 23.1 / 22.7; 899 KB: 30.7 / 26.0).
-constexpr int kGemvFullFromBytesI8 = 704 * 1024;
+// Integer path, piece table: one entry per k-tile and token: 3 pieces x 128 bytes, then 8 columns x 8 bytes of
+// column metadata (behind the pieces of the last token).
+constexpr int kGemvPieceEntryBytes = 512;
+// The table pays when a CTA's range passes over the same k-tiles at least this many times (in percent): filling it
+// costs the start of the call about as much as it saves on a range of 1.5 passes (4096 x 14336 on 148 SMs: 11.5 us
+// either way alone, 0.6 us slower inside the decode step).
+#ifndef TF_PIECE_TAB_MIN_REUSE_PCT
+#define TF_PIECE_TAB_MIN_REUSE_PCT 200
+#endif
+// Packed bytes per CTA from which the integer path uses the whole-SM configuration, and its consumer warps there.
+// A half-SM CTA has a ring of four 17 KB stages, and every tile a warp works on is a tile that is not in flight: eight
+// warps on int8 tiles (8.3 KB) hold the whole ring, on 4-bit tiles half of it.  The whole-SM form has a ring of nine
+// or ten stages; with about 66 KB of tiles in the warps' hands (8 warps on int8, 16 on 4-bit tiles) it streams long
+// ranges faster than the half-SM form, which wins on short ranges because the next GEMV's CTAs sit beside it with
+// their rings full.
+constexpr int kGemvFullFromBytesI8W4 = TF_I8_FULL_BYTES_W4;
+constexpr int kGemvFullFromBytesI8W8 = TF_I8_FULL_BYTES_W8;
+__host__ __device__ constexpr int gemv_i8_full_consumers(int bits) { return bits == 8 ? 8 : 16; }
 constexpr int kGemvMaxDevices = 64;            // devices the per-device caches cover
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
@@ -62,6 +88,7 @@ struct GemvPlan {
     int stages;        // ring depth
     bool full;         // whole-SM configuration
     bool i8;           // integer path: codes x activation pieces on the integer warp MMA (1 or 2 tokens)
+    int piece_tab;     // integer path: entries of the CTA-wide table of activation pieces (0 = every warp prepares its own tile's)
     int cluster;       // CTAs per cluster (1 = global mode: cut strips go through the workspace)
     int nclusters;     // cluster mode: number of clusters (grid = nclusters * cluster); global mode: CTAs that get tiles
     int xslot_bytes;   // cluster mode: bytes of one partial-sum slot in shared memory

@@ -29,14 +29,17 @@ def test_plan_invariants(bits, sm_count):
         p = tf.tf_gemv_plan(bits, M, K, N, sm_count)
         tiles = (K // 128) * (-(-N // 64))
         assert 1 <= p["grid"] <= 256 and p["grid"] <= max(sm_count, 1) or p["cluster"] > 1
-        assert p["threads"] == 32 * (p["consumers"] + 2) and 4 <= p["consumers"] <= 12
+        assert p["threads"] == 32 * (p["consumers"] + 2) and 4 <= p["consumers"] <= 16
         assert p["stages"] >= 2
         assert p["cluster"] in (1, 2, 4, 8)
         assert 1 <= p["nclusters"] <= max(p["grid"], 1)                  # CTAs (or clusters) that take part
         if M > 8:
             assert p["full"] == 1 and p["i8"] == 0 and p["consumers"] <= 8
         if M <= 2:
-            assert p["i8"] == 1                                          # both formats take the integer path at 1 and 2 tokens
+            assert p["i8"] in (1, 2)                                     # both formats take the integer path at 1 and 2 tokens
+            if p["i8"] == 2:                                             # piece table: only where a range passes over its k-tiles twice
+                per_cta = -(-tiles // p["nclusters"])
+                assert per_cta * 100 >= (K // 128) * 200
         else:
             assert p["i8"] == 0 and p["full"] == 1                       # the floating-point path takes the whole SM
         if p["cluster"] == 1 and tiles >= sm_count:
@@ -51,6 +54,15 @@ def test_plan_of_the_benchmark_shapes_on_a_b200():
         assert kind(tf.tf_gemv_plan(4, 4, K, N, 148)) == "whole"
     # no GPU here: the cluster-occupancy query fails, so 9..16 tokens plan for global mode
     assert kind(tf.tf_gemv_plan(4, 16, 4096, 14336, 148)) == "whole"
+    # long ranges of the integer path take the whole SM: 16 consumer warps on 4-bit tiles, 8 on int8 tiles
+    p = tf.tf_gemv_plan(4, 1, 4096, 32768, 148)
+    assert (p["full"], p["consumers"], p["i8"]) == (1, 16, 2)            # 111 tiles over 32 k-tiles: pieces prepared once per CTA
+    p = tf.tf_gemv_plan(8, 1, 4096, 14336, 148)
+    assert (p["full"], p["consumers"], p["i8"]) == (1, 8, 1)
+    assert tf.tf_gemv_plan(4, 2, 256, 32768, 148)["i8"] == 2 and tf.tf_gemv_plan(4, 2, 256, 32768, 148)["full"] == 0
+    for (K, N) in ((4096, 14336), (14336, 4096), (4096, 4096)):          # the decode step's shapes: half SM, no table
+        p = tf.tf_gemv_plan(4, 1, K, N, 148)
+        assert (p["full"], p["consumers"], p["i8"]) == (0, 8, 1)
     p = tf.tf_gemv_plan(4, 1, 4096, 1024, 148)
     assert p["grid"] == 148 and p["nclusters"] == 64                     # 64 CTAs x 8 tiles take part, the grid stays one per SM
     p = tf.tf_gemv_plan(4, 1, 4096, 4096, 148)

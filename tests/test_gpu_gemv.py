@@ -28,6 +28,21 @@ def test_gemv_w8_small(M, K, N):
     gu.check_against_oracle(p, gu.run(p, "gemv"))
 
 
+# ranges that pass over their k-tiles several times: the integer path prepares the activation pieces once per CTA
+PIECE_TABLE = [(1, 128, 8192), (2, 128, 8192), (1, 384, 30000), (2, 256, 32768), (1, 896, 30000), (2, 640, 20000), (1, 4096, 32768), (2, 4096, 32768)]
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("M,K,N", PIECE_TABLE)
+def test_gemv_integer_path_with_piece_table(bits, M, K, N):
+    if bits == 4 or K < 896:                # int8 tiles are twice the bytes: the larger shapes take the whole SM, where the table would cost a stage
+        assert tf.tf_gemv_plan(bits, M, K, N)["i8"] == 2
+    p = (wl.make_w4 if bits == 4 else wl.make_w8)(M, K, N, seed=M * 7 + K + N)
+    y = gu.run(p, "gemv")
+    gu.check_against_oracle(p, y)
+    assert np.array_equal(y, gu.run(p, "gemv"))
+
+
 @pytest.mark.parametrize("bits", [4, 8])
 def test_one_hot_activations_pick_exact_weights(bits):
     """a = e_k: y[n] must be bf16(w[k][n]) exactly (one rounding at the output, none on the weights)."""
