@@ -52,11 +52,10 @@ __device__ __forceinline__ void mma_s8_16832(int d[4], uint32_t a0, uint32_t a1,
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// The same with D = A . B (no accumulator to clear first).
-__device__ __forceinline__ void mma_s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    const int zero = 0;
+// The same with D = A . B + c in every element (no accumulator to set first).
+__device__ __forceinline__ void mma_s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1, int c) {
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c));
 }
 
 // The same shapes with unsigned bytes in the 16-row operand (4-bit codes 0..15 as they come out of a packed word).
@@ -64,16 +63,16 @@ __device__ __forceinline__ void mma_u8s8_16832(int d[4], uint32_t a0, uint32_t a
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void mma_u8s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    const int zero = 0;
+__device__ __forceinline__ void mma_u8s8_16832_first(int d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1, int c) {
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c));
 }
 
-// int -> float for |v| < 2^22 without the conversion unit: 1.5 * 2^23 + v is exact in fp32.
-__device__ __forceinline__ float small_int_to_float(int v) {
-    return __int_as_float(0x4B400000 + v) - 12582912.0f;
-}
+// int -> float for |v| < 2^22 without the conversion unit: the bits of the integer 0x4B400000 + v are the float
+// 1.5 * 2^23 + v, exactly.  The integer MMAs start their accumulators at kIntAsFloatBias, so a tile's sums come out of
+// the tensor pipe already in that form, and (f - 1.5 * 2^23) * c is one fused multiply-add with -1.5 * 2^23 * c.
+constexpr int kIntAsFloatBias = 0x4B400000;
+constexpr float kIntAsFloatBiasValue = 12582912.0f;
 
 __device__ __forceinline__ int range_start(int cta, int total, int grid) {
     return static_cast<int>((static_cast<long long>(cta) * total) / grid);
@@ -772,7 +771,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                                 // One AND per operand register instead of a shift and an AND: 32 instructions less per tile.
                                 const uint32_t a0 = x0 & 0x0F0F0F0Fu, a1 = x0 & 0xF0F0F0F0u;            // k-block 2i
                                 const uint32_t a2 = x1 & 0x0F0F0F0Fu, a3 = x1 & 0xF0F0F0F0u;            // k-block 2i + 1
-                                if (i == 0) mma_u8s8_16832_first(d[w], a0, a1, a2, a3, bw[0], bw[1]);
+                                if (i == 0) mma_u8s8_16832_first(d[w], a0, a1, a2, a3, bw[0], bw[1], kIntAsFloatBias);
                                 else mma_u8s8_16832(d[w], a0, a1, a2, a3, bw[2 * i], bw[2 * i + 1]);
                             }
                         }
@@ -795,7 +794,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                                 a[2 * hb] = __byte_perm(w0, w1, 0x5410);         // row g,   k 0..3 of this thread
                                 a[2 * hb + 1] = __byte_perm(w0, w1, 0x7632);     // row g+8
                             }
-                            if (i == 0) mma_s8_16832_first(d[w], a[0], a[1], a[2], a[3], bw[0], bw[1]);
+                            if (i == 0) mma_s8_16832_first(d[w], a[0], a[1], a[2], a[3], bw[0], bw[1], kIntAsFloatBias);
                             else mma_s8_16832(d[w], a[0], a[1], a[2], a[3], bw[2 * i], bw[2 * i + 1]);
                         }
                     }
@@ -817,14 +816,16 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                         mbar_arrive_n(empty0 + 8 * s, slot == tiles_here - 1 ? (uint32_t)(kR - tiles_here + 1) : 1u);
                     }
                     const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
+                    // d holds the bits of 1.5 * 2^23 + D: (that - 1.5 * 2^23) * column scale is one exact fused multiply-add
+                    const float off_x = -kIntAsFloatBiasValue * col_scale.x, off_y = -kIntAsFloatBiasValue * col_scale.y;
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
                         const float s_g = fp16_bits_to_float((uint16_t)(sw[w] & 0xFFFFu));
                         const float s_g8 = fp16_bits_to_float((uint16_t)(sw[w] >> 16)) * (BITS == 4 ? 0.0625f : 1.f);     // 4-bit: row g + 8 holds 16 (q - z)
-                        acc[w][0][0] = fmaf(small_int_to_float(d[w][0]) * col_scale.x, s_g, acc[w][0][0]);
-                        acc[w][0][1] = fmaf(small_int_to_float(d[w][1]) * col_scale.y, s_g, acc[w][0][1]);
-                        acc[w][0][2] = fmaf(small_int_to_float(d[w][2]) * col_scale.x, s_g8, acc[w][0][2]);
-                        acc[w][0][3] = fmaf(small_int_to_float(d[w][3]) * col_scale.y, s_g8, acc[w][0][3]);
+                        acc[w][0][0] = fmaf(fmaf(__int_as_float(d[w][0]), col_scale.x, off_x), s_g, acc[w][0][0]);
+                        acc[w][0][1] = fmaf(fmaf(__int_as_float(d[w][1]), col_scale.y, off_y), s_g, acc[w][0][1]);
+                        acc[w][0][2] = fmaf(fmaf(__int_as_float(d[w][2]), col_scale.x, off_x), s_g8, acc[w][0][2]);
+                        acc[w][0][3] = fmaf(fmaf(__int_as_float(d[w][3]), col_scale.y, off_y), s_g8, acc[w][0][3]);
                     }
                 } else {
                 // ---- floating-point path: group after group (one group per tile unless the group size is 64 or 32) ----
