@@ -219,97 +219,69 @@ __device__ __noinline__ bool gather_rows(float4* slot, int count, int M, float4 
 
 }  // namespace
 
-// Integer path, piece table: the activation pieces of the k-tiles of a CTA's range, prepared once.  Entry e holds
-// k-tile (t_first + e) mod ktiles: per token three piece columns of 32 words (the word of k-block kb and k quarter t at
-// t * 8 + kb, so that a thread of the MMA phase finds the eight k-blocks of its column and quarter in two 16-byte
-// loads), then 8 column entries {2^(emax-148) 256^j, sum of the piece over the tile}.  kLanes lanes prepare one
-// entry (lane u of the group holds kVals consecutive k), a warp 32 / kLanes entries per pass.  Not inlined: the
-// table is filled once per kernel, and inlined it took registers from the tile loop (spills that were reloaded per
-// tile: a whole-SM range of 111 tiles ran 0.5 us longer).
-template <int BITS, int kLanes>
-__device__ __noinline__ void fill_piece_table(uint32_t* pscr, const __nv_bfloat16* __restrict__ a_glob, int M, int K, int ktiles,
-                                              int T_first, int piece_n, int cw, int nconsumers, int lane) {
-    constexpr int kVals = 128 / kLanes, kPerPass = 32 / kLanes, kColWords = 32;
-    const int piece_entry_words = (kGemvPieceEntryBytes / 4) * M;
-    const int b = lane / kLanes, u = lane % kLanes;
-    for (int e0 = kPerPass * cw; e0 < piece_n; e0 += kPerPass * nconsumers) {
-        const int e = e0 + b;
-        const bool live = e < piece_n;
-        int T = T_first + e;                    // e < ktiles
-        if (T >= ktiles) T -= ktiles;
-        uint32_t* ent = pscr + (size_t)(live ? e : 0) * piece_entry_words;
-        uint2* meta = reinterpret_cast<uint2*>(ent + 96 * M);
+// Integer path: the activation pieces of one k-tile (up to two tokens), from the raw bf16 of lane L (k = 4L .. 4L+3).
+// dst: [column][kGemvPieceColWords] piece words, the word of lane L at (L & 3) * 8 + (L >> 2), so that a thread of the
+// MMA phase finds the eight k-blocks of its column and k quarter in two 16-byte loads (columns 36 words apart fall
+// into different banks); meta: [column] {2^(emax-148) 256^j, sum of the piece over the tile} in 8-byte entries, a
+// thread's two columns = one 16-byte load (with 4-byte entries and an 8-byte load the same kernel ran 12 % slower:
+// measured, cause not established).
+constexpr int kGemvPieceColWords = 36;
+template <int BITS>
+__device__ __forceinline__ void make_pieces(const uint2 (&raws)[2], uint32_t* dst, uint2* meta, int M, int lane) {
+    constexpr int kColWords = kGemvPieceColWords;
 #pragma unroll
-        for (int m = 0; m < 2; ++m) {
-            if (m < M) {
-                uint32_t x[kVals / 2];
-                const __nv_bfloat16* src = a_glob + (size_t)m * K + (size_t)T * kTileK + kVals * u;
-                if constexpr (kVals == 4) {
-                    uint2 r = make_uint2(0u, 0u);
-                    if (live) r = __ldcg(reinterpret_cast<const uint2*>(src));
-                    x[0] = r.x; x[1] = r.y;
-                } else {
+    for (int m = 0; m < 2; ++m) {
+        if (m < M) {
+            const uint2 raw = raws[m];
+            const uint32_t x0 = raw.x, x1 = raw.y;
+            uint32_t e = max(max((x0 << 17) >> 24, (x0 << 1) >> 24), max((x1 << 17) >> 24, (x1 << 1) >> 24));
+            e = __reduce_max_sync(0xFFFFFFFFu, e);
+            e = max(e, 22u);                                  // keeps both powers of two normal numbers
+            const float mult = __uint_as_float((275u - e) << 23);          // 2^(148 - emax)
+            // v + 0x808080 has the bytes p0 + 128, p1 + 128, p2 + 128 of the balanced split
+            uint32_t v[4];
+            v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
+            v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
+            v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
+            v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
+            // 4 x 3 byte transpose: one word per piece, bytes in the k order of the weight operand's bytes
+            // (int8: k, k+1, k+2, k+3; 4-bit: k, k+2, k+1, k+3, the order of a packed word's nibble pairs)
+            const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
+            const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
+            uint32_t word[3];
+            word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+            word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
+            word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
+            // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
+            const float se = e == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((e - 21u) << 23);
 #pragma unroll
-                    for (int i = 0; i < kVals / 8; ++i) {
-                        uint4 r = make_uint4(0u, 0u, 0u, 0u);
-                        if (live) r = __ldcg(reinterpret_cast<const uint4*>(src) + i);
-                        x[4 * i] = r.x; x[4 * i + 1] = r.y; x[4 * i + 2] = r.z; x[4 * i + 3] = r.w;
-                    }
-                }
-                uint32_t ex = 0u;
-#pragma unroll
-                for (int i = 0; i < kVals / 2; ++i) ex = max(ex, max((x[i] << 17) >> 24, (x[i] << 1) >> 24));
-#pragma unroll
-                for (int d = 1; d < kLanes; d *= 2) ex = max(ex, __shfl_xor_sync(0xFFFFFFFFu, ex, d));
-                ex = max(ex, 22u);                                    // keeps both powers of two normal numbers
-                const float mult = __uint_as_float((275u - ex) << 23);                // 2^(148 - emax)
-                // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
-                const float se = ex == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((ex - 21u) << 23);
-                int psum[3] = {0, 0, 0};
-#pragma unroll
-                for (int q = 0; q < kVals / 4; ++q) {           // four consecutive k: one word per piece
-                    const int k0 = kVals * u + 4 * q;           // k-block k0 / 16, k quarter (k0 % 16) / 4
-                    const uint32_t x0 = x[2 * q], x1 = x[2 * q + 1];
-                    uint32_t v[4];
-                    v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
-                    v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
-                    v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
-                    v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
-                    const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
-                    const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
-                    uint32_t word[3];
-                    word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
-                    word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
-                    word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) {
-                        if (live) ent[(3 * m + j) * kColWords + ((k0 >> 2) & 3) * 8 + (k0 >> 4)] = word[j];
-                        if constexpr (BITS == 4) psum[j] = __dp4a((int)word[j], 0x01010101, psum[j]);
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 3; ++j) {
-                    if constexpr (BITS == 4) {                  // sum of the piece over the tile's 128 k, for the zero point
-#pragma unroll
-                        for (int d = 1; d < kLanes; d *= 2) psum[j] += __shfl_xor_sync(0xFFFFFFFFu, psum[j], d);
-                    }
-                    if (live && u == 0)
-                        meta[3 * m + j] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum[j]);
-                }
+            for (int j = 0; j < 3; ++j) {
+                const int c = 3 * m + j;
+                dst[c * kColWords + (lane & 3) * 8 + (lane >> 2)] = word[j];
+                int psum = 0;                           // 4-bit: sum of the piece over the tile's 128 k, for the zero point
+                if constexpr (BITS == 4) psum = __reduce_add_sync(0xFFFFFFFFu, __dp4a((int)word[j], 0x01010101, 0));
+                if (lane == 0) meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum);
             }
         }
-        if (live && u == 0) {                           // columns without a token contribute nothing
-#pragma unroll
-            for (int c = 3; c < 8; ++c)
-                if (c >= 3 * M) meta[c] = make_uint2(0u, 0u);
-        }
     }
+    if (lane == 0) {                                    // columns without a token contribute nothing
+#pragma unroll
+        for (int c = 3; c < 8; ++c)
+            if (c >= 3 * M) meta[c] = make_uint2(0u, 0u);
+    }
+}
+// The same as a call: where pieces are prepared on the first visit of a k-tile only, the code stays out of the tile
+// loop's register allocation.
+template <int BITS>
+__device__ __noinline__ void make_pieces_call(const uint2 (&raws)[2], uint32_t* dst, uint2* meta, int M, int lane) {
+    make_pieces<BITS>(raws, dst, meta, M, lane);
 }
 
 // G = groups per tile: 1 for group sizes that are multiples of 128, 2 / 4 for the 4-bit group sizes 64 / 32.
-// I8 = 0: floating-point path; 1: integer path, every consumer warp prepares the activation pieces of the tile it
-// works on; 2: integer path, the consumer warps prepare the pieces of every k-tile of the CTA's range once, before
-// the first tile, into a table all of them read (ranges that pass over the same k-tiles several times).
+// I8 = 0: floating-point path; 1: integer path, a consumer warp prepares the activation pieces of every tile it works
+// on; 2: integer path for ranges that pass over the same k-tiles more than once, with K a multiple of 128 times the
+// number of consumer warps: a warp then meets the same k-tiles on every pass, prepares the pieces of a k-tile on its
+// first visit and keeps them (piece table, one entry per k-tile, each entry written and read by one warp only).
 template <int BITS, int MT, bool FULL, bool CL, int I8, int G = 1>
 __global__ void __launch_bounds__(gemv_max_threads(MT, FULL, I8 != 0), FULL ? 1 : 2)
 gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __restrict__ a_glob, __nv_bfloat16* __restrict__ y, int M, int K, int N, int ktiles, int total_tiles,
@@ -474,10 +446,14 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 float4 sum[kVec];
 #pragma unroll
                 for (int e = 0; e < kVec; ++e) sum[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                // (the integer path has at most two tokens, one row pair: a quarter of the loads and additions of this
+                // loop, which for the last segment of a range is the tail of the kernel; a run-time bound on the row
+                // pairs for the other paths made them slower: 36.7 against 35.7 us over the four shapes at 4 tokens)
+                constexpr int kVecUsed = I8 ? 1 : kVec;
                 for (int w = 0; w < nconsumers; ++w) {
                     const float4* src = reinterpret_cast<const float4*>(red + (size_t)(rb * nconsumers + w) * kRedWarp) + lane;
 #pragma unroll
-                    for (int e = 0; e < kVec; ++e) {
+                    for (int e = 0; e < kVecUsed; ++e) {
                         const float4 v = src[32 * e];
                         sum[e].x += v.x; sum[e].y += v.y; sum[e].z += v.z; sum[e].w += v.w;
                     }
@@ -541,70 +517,15 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         auto load_ag_kb = [&](const __nv_bfloat16* base, int kb) {
             if (g < M) ag[0][kRegActs ? kb : 0] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)g * K + 4 * t + 16 * kb));
         };
-        // Integer path: the activation pieces of one (k-tile, token) pair, from the raw bf16 of lane L (k = 4L .. 4L+3).
-        // dst: [column][kColWords] piece words, the word of lane L at (L & 3) * 8 + (L >> 2), so that a thread of the
-        // MMA phase finds the eight k-blocks of its column and k quarter in two 16-byte loads; meta: [column]
-        // {2^(emax-148) 256^j, sum of the piece over the tile} in 8-byte entries, a thread's two columns = one 16-byte
-        // load (with 4-byte entries and an 8-byte load the same kernel ran 12 % slower: measured, cause not established).
-        constexpr int kColWords = I8 == 2 ? 32 : 36;
-        auto make_pieces = [&](const uint2 (&raws)[2], uint32_t* dst, uint2* meta) {
-#pragma unroll
-            for (int m = 0; m < 2; ++m) {
-                if (m < M) {
-                    const uint2 raw = raws[m];
-                    const uint32_t x0 = raw.x, x1 = raw.y;
-                    uint32_t e = max(max((x0 << 17) >> 24, (x0 << 1) >> 24), max((x1 << 17) >> 24, (x1 << 1) >> 24));
-                    e = __reduce_max_sync(0xFFFFFFFFu, e);
-                    e = max(e, 22u);                                  // keeps both powers of two normal numbers
-                    const float mult = __uint_as_float((275u - e) << 23);          // 2^(148 - emax)
-                    // v + 0x808080 has the bytes p0 + 128, p1 + 128, p2 + 128 of the balanced split
-                    uint32_t v[4];
-                    v[0] = (uint32_t)__float2int_rn(__uint_as_float(x0 << 16) * mult) + 0x808080u;
-                    v[1] = (uint32_t)__float2int_rn(__uint_as_float(x0 & 0xFFFF0000u) * mult) + 0x808080u;
-                    v[2] = (uint32_t)__float2int_rn(__uint_as_float(x1 << 16) * mult) + 0x808080u;
-                    v[3] = (uint32_t)__float2int_rn(__uint_as_float(x1 & 0xFFFF0000u) * mult) + 0x808080u;
-                    // 4 x 3 byte transpose: one word per piece, bytes in the k order of the weight operand's bytes
-                    // (int8: k, k+1, k+2, k+3; 4-bit: k, k+2, k+1, k+3, the order of a packed word's nibble pairs)
-                    const uint32_t ab01 = __byte_perm(v[0], v[1], 0x5140), ab2 = __byte_perm(v[0], v[1], 0x0062);
-                    const uint32_t cd01 = __byte_perm(v[2], v[3], 0x5140), cd2 = __byte_perm(v[2], v[3], 0x0062);
-                    uint32_t word[3];
-                    word[0] = __byte_perm(ab01, cd01, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
-                    word[1] = __byte_perm(ab01, cd01, BITS == 8 ? 0x7632 : 0x7362) ^ 0x80808080u;
-                    word[2] = __byte_perm(ab2, cd2, BITS == 8 ? 0x5410 : 0x5140) ^ 0x80808080u;
-                    // 2^(emax - 148); an Inf or NaN among the 128 activations makes this token's outputs NaN
-                    const float se = e == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((e - 21u) << 23);
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) {
-                        const int c = 3 * m + j;
-                        dst[c * kColWords + (lane & 3) * 8 + (lane >> 2)] = word[j];
-                        int psum = 0;                           // 4-bit: sum of the piece over the tile's 128 k, for the zero point
-                        if constexpr (BITS == 4) psum = __reduce_add_sync(0xFFFFFFFFu, __dp4a((int)word[j], 0x01010101, 0));
-                        if (lane == 0) meta[c] = make_uint2(__float_as_uint(se * (j == 0 ? 1.f : j == 1 ? 256.f : 65536.f)), (uint32_t)psum);
-                    }
-                }
-            }
-            if (lane == 0) {                                    // columns without a token contribute nothing
-#pragma unroll
-                for (int c = 3; c < 8; ++c)
-                    if (c >= 3 * M) meta[c] = make_uint2(0u, 0u);
-            }
-        };
+        constexpr int kColWords = kGemvPieceColWords;
         grid_dependency_wait();                         // the activations belong to earlier kernels until now
-        // Piece table: entry e holds k-tile (t0 + e) mod ktiles, so local tile j of the range finds its pieces in
-        // entry j mod piece_n, piece_n = min(ntiles, ktiles).  kLanes lanes prepare one entry (lane u of the group holds
-        // kVals consecutive k), a warp 32 / kLanes entries per pass, so that the 32 k-tiles of K = 4096 are one pass of
-        // all consumer warps (8 warps x 4 entries in the half-SM form, 16 x 2 in the whole-SM form); then the consumer
-        // warps meet.  (One entry per warp and pass, four passes one after the other, took about 1 us in the half-SM
-        // form: more than the table saved on a range of 48 tiles.)
+        // Piece table (I8 == 2): local tile j of the range finds its pieces in entry j mod piece_n, piece_n =
+        // min(ntiles, ktiles); j < piece_n is the first visit of that k-tile.  ktiles is a multiple of the number of
+        // consumer warps, so tiles j and j + ktiles belong to the same warp: no warp reads another warp's entry.
         const int piece_entry_words = (kGemvPieceEntryBytes / 4) * M;
         const int piece_n = min(ntiles, ktiles);
         const int T_first = t0 % ktiles;                // k-tile index of the range's first tile
-        int piece_e = 0;
-        if constexpr (I8 == 2) {
-            fill_piece_table<BITS, FULL ? 16 : 8>(pscr, a_glob, M, K, ktiles, T_first, piece_n, cw, nconsumers, lane);
-            asm volatile("bar.sync 1, %0;" ::"r"(nconsumers * 32) : "memory");
-            if (piece_n > 0) piece_e = cw % piece_n;
-        }
+        int piece_e = cw;                               // entry of this warp's next tile (cw < piece_n whenever it has one)
         if constexpr (kRegActs) {
 #pragma unroll
             for (int kb = 0; kb < 8; ++kb) ag[0][kb] = make_uint2(0u, 0u);
@@ -638,8 +559,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
         int abuf_cur = 0;
         if (kAhead && cw < ntiles) {
             const __nv_bfloat16* base = a_glob + (size_t)T_act * kTileK;
-            if constexpr (I8 == 1) load_araw(base);
-            else if constexpr (I8 == 0) {
+            if constexpr (I8 != 0) load_araw(base);
+            else {
 #pragma unroll
                 for (int kb = 0; kb < 8; ++kb) load_ag_kb(base, kb);
             }
@@ -731,13 +652,24 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                     const uint32_t* scr;                                // this tile's piece words and column metadata
                     const uint2* col_meta;
                     if constexpr (I8 == 2) {
-                        scr = pscr + piece_e * piece_entry_words;
-                        col_meta = reinterpret_cast<const uint2*>(scr + 96 * M);
+                        uint32_t* ent = pscr + piece_e * piece_entry_words;
+                        uint2* ent_meta = reinterpret_cast<uint2*>(ent + 3 * kColWords * M);
                         piece_e += nconsumers;                          // the warp's next tile is nconsumers k-tiles further
                         while (piece_e >= piece_n) piece_e -= piece_n;
+                        if (j < piece_n) {                              // first visit of this k-tile
+                            // (as a call in the whole-SM form with its 96 registers: inlined it spilled inside the tile loop,
+                            // 17.8 against 17.1 us on 1x4096x32768; inlined in the half-SM form, where the call was the
+                            // slower one, 12.0 against 10.9 us on 1x4096x14336)
+                            if constexpr (FULL) make_pieces_call<BITS>(araw, ent, ent_meta, M, lane);
+                            else make_pieces<BITS>(araw, ent, ent_meta, M, lane);
+                            if (j + nconsumers < piece_n) load_araw(next_base);    // later visits need no activations
+                            __syncwarp();
+                        }
+                        scr = ent;
+                        col_meta = ent_meta;
                     } else {
                         uint32_t* mine_scr = pscr + cw * 256;
-                        make_pieces(araw, mine_scr, reinterpret_cast<uint2*>(mine_scr + 216));
+                        make_pieces<BITS>(araw, mine_scr, reinterpret_cast<uint2*>(mine_scr + 216), M, lane);
                         scr = mine_scr;
                         col_meta = reinterpret_cast<const uint2*>(mine_scr + 216);
                         if (has_next) load_araw(next_base);             // the next tile's activations, under this tile's MMAs
@@ -1138,18 +1070,18 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // no more stages than the range has chunks
     const int chunks = (tiles_per_cta + kr - 1) / kr + 2;
     if (stages > chunks) stages = chunks;
-    // Integer path: a range that passes over the same k-tiles several times prepares the activation pieces of each
-    // k-tile once per CTA instead of once per tile, if the table costs the ring no stage.
+    // Integer path: where a range passes over the same k-tiles more than once and K is a multiple of 128 x consumer
+    // warps, every warp meets the same k-tiles on each pass and keeps the activation pieces it has prepared (one table
+    // entry per k-tile instead of one scratch entry per warp), if that costs the ring no stage.
+    // (int8 weights, whole SM, 4096x28672 and 4096x32768: with a table and one ring stage less 22.4 / 24.7 us, without 21.1 / 23.6)
     p.piece_tab = 0;
-    if (p.i8) {
-        const int entries = tiles_per_cta < p.ktiles ? tiles_per_cta : p.ktiles;
-        const int table = (entries * kGemvPieceEntryBytes * M + 1023) / 1024 * 1024;
+    if (p.i8 && tiles_per_cta >= p.ktiles + p.consumers && p.ktiles % p.consumers == 0) {
+        const int table = (p.ktiles * kGemvPieceEntryBytes * M + 1023) / 1024 * 1024;
         int with = (gemv_smem_budget(mt, p.full) - (base + table)) / p.stage_bytes;
         if (with > kGemvMaxStages) with = kGemvMaxStages;
         if (with > chunks) with = chunks;
-        // (int8 weights, whole SM, 4096x28672 and 4096x32768: with the table and one ring stage less 22.4 / 24.7 us, without 21.1 / 23.6)
-        if (with >= stages && tiles_per_cta * 100 >= p.ktiles * TF_PIECE_TAB_MIN_REUSE_PCT) {
-            p.piece_tab = entries;
+        if (with >= stages) {
+            p.piece_tab = p.ktiles;
             fixed = base + table;
         }
     }

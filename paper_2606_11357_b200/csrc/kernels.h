@@ -18,8 +18,9 @@ namespace tf {
 //   integer path (1 and 2 tokens), short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs
 //     fit beside this one's and have their rings full of weights when this kernel completes.
 //   integer path, long ranges: the whole SM, a ring of seven to ten stages, and as many consumer warps as hold
-//     about 66 KB of tiles (16 on 4-bit tiles, 8 on int8 tiles); where the range passes over the same k-tiles at
-//     least twice the activation pieces are prepared once per CTA (piece table) instead of once per tile.
+//     about 66 KB of tiles (16 on 4-bit tiles, 8 on int8 tiles).
+//   Either form: where a range passes over its k-tiles more than once and K is a multiple of 128 x consumer warps,
+//     a warp keeps the activation pieces of the k-tiles it has visited (piece table) instead of preparing them per tile.
 //   floating-point path up to 8 tokens: the whole SM, 12 consumer warps and a ring deep enough to keep HBM busy
 //     while 12 tiles are being consumed.  A consumer warp
 //     of the floating-point path is bound by instruction issue (about 20 issue cycles per packed word of 8
@@ -36,15 +37,9 @@ __host__ __device__ constexpr int gemv_smem_budget(int mt, bool full) { return (
 // Shared memory a half-SM CTA asks for when two of its kind must not share an SM: with 228 KB per SM and 1 KB reserved
 // per CTA, two of these do not fit (2 x 115 KB), one beside a plain half-SM CTA (at most 110 KB) does.
 constexpr int kGemvSoloSmemBytes = 114 * 1024;
-// Integer path, piece table: one entry per k-tile and token: 3 pieces x 128 bytes, then 8 columns x 8 bytes of
-// column metadata (behind the pieces of the last token).
+// Integer path, piece table: one entry per k-tile: per token 3 piece columns of 36 words (32 used; the padding keeps
+// the columns in different banks), then 8 columns x 8 bytes of column metadata; 512 bytes per token.
 constexpr int kGemvPieceEntryBytes = 512;
-// The table pays when a CTA's range passes over the same k-tiles at least this many times (in percent): filling it
-// costs the start of the call about as much as it saves on a range of 1.5 passes (4096 x 14336 on 148 SMs: 11.5 us
-// either way alone, 0.6 us slower inside the decode step).
-#ifndef TF_PIECE_TAB_MIN_REUSE_PCT
-#define TF_PIECE_TAB_MIN_REUSE_PCT 200
-#endif
 // Packed bytes per CTA from which the integer path uses the whole-SM configuration, and its consumer warps there.
 // A half-SM CTA has a ring of four 17 KB stages, and every tile a warp works on is a tile that is not in flight: eight
 // warps on int8 tiles (8.3 KB) hold the whole ring, on 4-bit tiles half of it.  The whole-SM form has a ring of nine

@@ -37,9 +37,9 @@ def test_plan_invariants(bits, sm_count):
             assert p["full"] == 1 and p["i8"] == 0 and p["consumers"] <= 8
         if M <= 2:
             assert p["i8"] in (1, 2)                                     # both formats take the integer path at 1 and 2 tokens
-            if p["i8"] == 2:                                             # piece table: only where a range passes over its k-tiles twice
+            if p["i8"] == 2:                                             # piece table: a warp meets the same k-tiles on every pass
                 per_cta = -(-tiles // p["nclusters"])
-                assert per_cta * 100 >= (K // 128) * 200
+                assert (K // 128) % p["consumers"] == 0 and per_cta >= K // 128 + p["consumers"]
         else:
             assert p["i8"] == 0 and p["full"] == 1                       # the floating-point path takes the whole SM
         if p["cluster"] == 1 and tiles >= sm_count:
@@ -56,13 +56,15 @@ def test_plan_of_the_benchmark_shapes_on_a_b200():
     assert kind(tf.tf_gemv_plan(4, 16, 4096, 14336, 148)) == "whole"
     # long ranges of the integer path take the whole SM: 16 consumer warps on 4-bit tiles, 8 on int8 tiles
     p = tf.tf_gemv_plan(4, 1, 4096, 32768, 148)
-    assert (p["full"], p["consumers"], p["i8"]) == (1, 16, 2)            # 111 tiles over 32 k-tiles: pieces prepared once per CTA
+    assert (p["full"], p["consumers"], p["i8"]) == (1, 16, 2)            # 111 tiles over 32 k-tiles: a warp keeps the pieces it has prepared
     p = tf.tf_gemv_plan(8, 1, 4096, 14336, 148)
-    assert (p["full"], p["consumers"], p["i8"]) == (1, 8, 1)
-    assert tf.tf_gemv_plan(4, 2, 256, 32768, 148)["i8"] == 2 and tf.tf_gemv_plan(4, 2, 256, 32768, 148)["full"] == 0
-    for (K, N) in ((4096, 14336), (14336, 4096), (4096, 4096)):          # the decode step's shapes: half SM, no table
+    assert (p["full"], p["consumers"], p["i8"]) == (1, 8, 1)             # int8, whole SM: a table would cost a ring stage
+    # the decode step's shapes take half an SM; 48 tiles over 32 k-tiles keep their pieces, 24 over 112 and 16 over 32 have none to keep
+    assert [tf.tf_gemv_plan(4, 1, K, N, 148)["i8"] for (K, N) in ((4096, 14336), (14336, 4096), (4096, 4096))] == [2, 1, 1]
+    for (K, N) in ((4096, 14336), (14336, 4096), (4096, 4096)):
         p = tf.tf_gemv_plan(4, 1, K, N, 148)
-        assert (p["full"], p["consumers"], p["i8"]) == (0, 8, 1)
+        assert (p["full"], p["consumers"]) == (0, 8)
+    assert tf.tf_gemv_plan(4, 1, 4096 + 128, 14336, 148)["i8"] == 1      # 33 k-tiles over 8 warps: a warp would meet other k-tiles on its second pass
     p = tf.tf_gemv_plan(4, 1, 4096, 1024, 148)
     assert p["grid"] == 148 and p["nclusters"] == 64                     # 64 CTAs x 8 tiles take part, the grid stays one per SM
     p = tf.tf_gemv_plan(4, 1, 4096, 4096, 148)

@@ -57,7 +57,7 @@ CHAINS = [
     ((4096, 14336, 4096), 16, ("whole", "whole")),
     ((4096, 4096, 1024), 16, ("cluster", "cluster")),
     ((4096, 32768, 1024), 2, ("whole", "half")),            # a long integer-path range: whole SM, 16 warps, piece table
-    ((256, 32768, 1024), 2, ("half", "half")),             # two tokens with the CTA-wide piece table, then without
+    ((1024, 32768, 1024), 2, ("half", "half")),            # two tokens with the piece table, then without
     ((384, 14336, 4096), 1, ("half", "half")),
 ]
 
