@@ -293,7 +293,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     constexpr int kR = gemv_chunk_tiles(BITS);            // tiles per bulk copy / ring stage
     constexpr int kTok = 8 * MT;
     constexpr int kVecPerKb = BITS == 4 ? 1 : 2;
-    constexpr int kRedWarp = kTok * kTileN;               // floats one consumer warp drops per strip segment
+    constexpr int kRedWarp = (I8 ? 2 : kTok) * kTileN;    // floats one consumer warp drops per strip segment (integer path: two token rows)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -872,6 +872,7 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     const int tok = 8 * mt + 2 * t;
+                    if (I8 && t != 0) continue;                 // integer path: tokens 0 and 1 sit in the t = 0 threads, the buffer has two rows
                     mine[tok * kTileN + 16 * w + g] = acc[w][mt][0];
                     mine[(tok + 1) * kTileN + 16 * w + g] = acc[w][mt][1];
                     mine[tok * kTileN + 16 * w + g + 8] = acc[w][mt][2];
@@ -1062,7 +1063,7 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // two buffers for the consumer warps' partial sums where the whole SM is taken (a boundary between strips then
     // costs a fast warp nothing; measured below), one in the half-SM form, where the second would cost a ring stage
     p.nred = p.full ? 2 : 1;
-    const int base = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.nred * p.consumers * 8 * mt * kTileN * 4 +
+    const int base = 1024 /*alignment slack*/ + kGemvBarrierBytes + p.nred * p.consumers * (p.i8 ? 2 : 8 * mt) * kTileN * 4 +
                      (p.cluster * p.xslot_bytes + 1023) / 1024 * 1024 + (mt == 2 ? p.consumers * kGemvActWarpBytes : 0);
     int fixed = base + (p.i8 ? p.consumers * 1024 : 0);
     int stages = (gemv_smem_budget(mt, p.full) - fixed) / p.stage_bytes;
@@ -1070,12 +1071,15 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // no more stages than the range has chunks
     const int chunks = (tiles_per_cta + kr - 1) / kr + 2;
     if (stages > chunks) stages = chunks;
+    // whole-SM integer path: a ring deeper than eight stages was slower (1x4096x32768 4-bit: 17.0 / 16.9 / 17.5 us with
+    // 6 / 8 / 10 stages; int8 1x4096x14336: 12.8 / 12.5 / 12.7 us with 6 / 8 / 11)
+    if (p.i8 && p.full && stages > kGemvI8FullMaxStages) stages = kGemvI8FullMaxStages;
     // Integer path: where a range passes over the same k-tiles more than once and K is a multiple of 128 x consumer
     // warps, every warp meets the same k-tiles on each pass and keeps the activation pieces it has prepared (one table
     // entry per k-tile instead of one scratch entry per warp), if that costs the ring no stage.
-    // (int8 weights, whole SM, 4096x28672 and 4096x32768: with a table and one ring stage less 22.4 / 24.7 us, without 21.1 / 23.6)
     p.piece_tab = 0;
-    if (p.i8 && tiles_per_cta >= p.ktiles + p.consumers && p.ktiles % p.consumers == 0) {
+    // (4-bit weights only: on int8 tiles, whole SM, the table was the slower form, 13.1 against 12.5 us on 1x4096x14336)
+    if (p.i8 && bits == 4 && tiles_per_cta >= p.ktiles + p.consumers && p.ktiles % p.consumers == 0) {
         const int table = (p.ktiles * kGemvPieceEntryBytes * M + 1023) / 1024 * 1024;
         int with = (gemv_smem_budget(mt, p.full) - (base + table)) / p.stage_bytes;
         if (with > kGemvMaxStages) with = kGemvMaxStages;

@@ -37,7 +37,7 @@ PIECE_TABLE = [(1, 1024, 30000), (2, 1024, 30000), (1, 2048, 32768), (2, 2048, 2
 @pytest.mark.parametrize("bits", [4, 8])
 @pytest.mark.parametrize("M,K,N", PIECE_TABLE)
 def test_gemv_integer_path_with_piece_table(bits, M, K, N):
-    if bits == 4:                               # int8 tiles are twice the bytes: other plans, some without the table
+    if bits == 4:                               # int8 weights prepare their pieces per tile
         assert tf.tf_gemv_plan(bits, M, K, N)["i8"] == 2
     p = (wl.make_w4 if bits == 4 else wl.make_w8)(M, K, N, seed=M * 7 + K + N)
     y = gu.run(p, "gemv")
