@@ -1074,6 +1074,12 @@ GemvPlan plan_gemv(int bits, int M, int K, int N, int sm_count, int groups) {
     // whole-SM integer path: a ring deeper than eight stages was slower (1x4096x32768 4-bit: 17.0 / 16.9 / 17.5 us with
     // 6 / 8 / 10 stages; int8 1x4096x14336: 12.8 / 12.5 / 12.7 us with 6 / 8 / 11)
     if (p.i8 && p.full && stages > kGemvI8FullMaxStages) stages = kGemvI8FullMaxStages;
+    // floating-point path up to 8 tokens on 4-bit tiles: five stages (three in the hands of the 12 consumer warps, two in
+    // flight).  Measured at 4 tokens with 4 / 5 / 6 / 7 / 9 stages: 4096x14336 12.2 / 11.6 / 11.7 / 11.9 / 12.3 us,
+    // 4096x32768 20.9 / 19.8 / 19.9 / 20.1 / 20.5 us; int8 tiles (six stages in the warps' hands) want the deep ring:
+    // 4096x14336 19.6 / 18.4 / 17.4 / 16.6 / 16.0 us.  (Why a deeper ring is slower on 4-bit tiles was not established;
+    // the consumers, not HBM, set the pace of this path.)
+    if (!p.i8 && mt == 1 && bits == 4 && stages > kGemvFpW4MaxStages) stages = kGemvFpW4MaxStages;
     // Integer path: where a range passes over the same k-tiles more than once and K is a multiple of 128 x consumer
     // warps, every warp meets the same k-tiles on each pass and keeps the activation pieces it has prepared (one table
     // entry per k-tile instead of one scratch entry per warp), if that costs the ring no stage.

@@ -50,6 +50,7 @@ constexpr int kGemvFullFromBytesI8W4 = TF_I8_FULL_BYTES_W4;
 constexpr int kGemvFullFromBytesI8W8 = TF_I8_FULL_BYTES_W8;
 __host__ __device__ constexpr int gemv_i8_full_consumers(int bits) { return bits == 8 ? 8 : 16; }
 constexpr int kGemvI8FullMaxStages = 8;
+constexpr int kGemvFpW4MaxStages = 5;
 constexpr int kGemvMaxDevices = 64;            // devices the per-device caches cover
 constexpr int kGemvMaxStages = 48;
 constexpr int kGemvBarrierBytes = 4096;       // 2 x 48 mbarriers + flags, then contributor offsets
