@@ -20,7 +20,9 @@ LIMIT_KCYCLES = 2000            # about 1 ms at 1.9 GHz
 # (kind, bits, M, K, N): the integer GEMV path, the floating-point GEMV path (whole SM), 9..16 tokens in global
 # mode and in cluster mode, the int8 GEMV, and the GEMM with a narrow and a full token tile (one of them cut between CTAs)
 CASES = [("gemv", 4, 1, 2048, 1024), ("gemv", 4, 5, 2048, 1024), ("gemv", 4, 16, 4096, 14336), ("gemv", 4, 16, 4096, 1024),
-         ("gemv", 8, 2, 1024, 512), ("gemm", 4, 24, 1024, 512), ("gemm", 4, 300, 2048, 1096), ("gemm", 8, 64, 512, 256)]
+         ("gemv", 8, 2, 1024, 512), ("gemm", 4, 24, 1024, 512), ("gemm", 4, 300, 2048, 1096), ("gemm", 8, 64, 512, 256),
+         # long integer-path ranges: whole SM with 16 consumer warps and the piece table (4-bit), with 8 warps (int8)
+         ("gemv", 4, 1, 4096, 32768), ("gemv", 8, 2, 4096, 14336)]
 
 
 @pytest.fixture(autouse=True)
