@@ -449,7 +449,11 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 // (the integer path has at most two tokens, one row pair: a quarter of the loads and additions of this
                 // loop, which for the last segment of a range is the tail of the kernel; a run-time bound on the row
                 // pairs for the other paths made them slower: 36.7 against 35.7 us over the four shapes at 4 tokens)
+                // Four warps' loads in flight at a time: this loop is the tail of every CTA (the last segment's sum sits
+                // between the last consumer warp and the store), and rolled up it cost the decode step 1.8 us (115.7 ->
+                // 113.9; unrolled by 2: 115.3, by 8: 114.7).
                 constexpr int kVecUsed = I8 ? 1 : kVec;
+#pragma unroll 4
                 for (int w = 0; w < nconsumers; ++w) {
                     const float4* src = reinterpret_cast<const float4*>(red + (size_t)(rb * nconsumers + w) * kRedWarp) + lane;
 #pragma unroll
