@@ -358,8 +358,9 @@ size_t tf_gemv_awq_raw_workspace_size(int M, int K, int N, int group_size);
  * 4.4 maps work to cores statically; here the mapping depends on the shape, and tests assert which one they hit).
  *   sm_count  SMs to plan for; <= 0 = the current device (then TF_ERR_ARCH / TF_ERR_CUDA as for a compute call).
  *   out       host, 8 ints: persistent CTAs, threads per CTA, consumer warps, ring stages, whole-SM CTA (1) or
- *             half-SM (0), integer path (1/0), CTAs per cluster (1 = cut strips go through the workspace), and
- *             the number of clusters (cluster mode) or of CTAs that get tiles (otherwise).
+ *             half-SM (0), integer path (0 = no, 1 = activation pieces prepared per tile, 2 = kept per k-tile
+ *             in a table), CTAs per cluster (1 = cut strips go through the workspace), and the number of clusters
+ *             (cluster mode) or of CTAs that get tiles (otherwise).
  * Pure host code apart from the device query; launches nothing.  Errors: TF_ERR_NULL, TF_ERR_SHAPE.
  */
 tf_status tf_gemv_plan(int bits, int M, int K, int N, int sm_count, int* out);
