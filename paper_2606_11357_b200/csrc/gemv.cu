@@ -525,7 +525,6 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             if (g < M) ag[0][kRegActs ? kb : 0] = __ldcg(reinterpret_cast<const uint2*>(base + (size_t)g * K + 4 * t + 16 * kb));
         };
         constexpr int kColWords = kGemvPieceColWords;
-        grid_dependency_wait();                         // the activations belong to earlier kernels until now
         // Piece table (I8 == 2): local tile j of the range finds its pieces in entry j mod piece_n, piece_n =
         // min(ntiles, ktiles); j < piece_n is the first visit of that k-tile.  ktiles is a multiple of the number of
         // consumer warps, so tiles j and j + ktiles belong to the same warp: no warp reads another warp's entry.
@@ -561,6 +560,10 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 if (row >= M) reinterpret_cast<uint4*>(my_abuf)[idx] = make_uint4(0u, 0u, 0u, 0u);
             }
             __syncwarp();
+        }
+        // Everything above touches registers and this CTA's shared memory only; from here on the warp reads activations.
+        grid_dependency_wait();                         // the activations belong to earlier kernels until now
+        if constexpr (kStaged) {
             if (cw < ntiles) stage_acts(a_glob + (size_t)T_act * kTileK, 0);
         }
         int abuf_cur = 0;
