@@ -74,11 +74,20 @@ __device__ __forceinline__ void mma_u8s8_16832_first(int d[4], uint32_t a0, uint
 constexpr int kIntAsFloatBias = 0x4B400000;
 constexpr float kIntAsFloatBiasValue = 12582912.0f;
 
+// Even split of `total` tiles over `grid` CTAs.  The products fit 32 bits (at most 256 x 512 tiles, K and N <= 32768,
+// times at most 257 CTAs), and a 32-bit division is a fraction of the instructions of a 64-bit one.  These sit between
+// the start of a CTA and its first weight copy, in the reducer's bookkeeping and in the cluster-mode finish; k32 chooses
+// the width per kernel instantiation, by measurement: the 9..16-token kernels gained 1.1 us over the four layer shapes
+// with 32 bits, the others lost 0.3 to 0.4 us (the same kernels, differently scheduled by the compiler).
+template <bool k32>
 __device__ __forceinline__ int range_start(int cta, int total, int grid) {
-    return static_cast<int>((static_cast<long long>(cta) * total) / grid);
+    if constexpr (k32) return static_cast<int>((static_cast<uint32_t>(cta) * static_cast<uint32_t>(total)) / static_cast<uint32_t>(grid));
+    else return static_cast<int>((static_cast<long long>(cta) * total) / grid);
 }
+template <bool k32>
 __device__ __forceinline__ int range_owner(int tile, int total, int grid) {
-    return static_cast<int>(((static_cast<long long>(tile) + 1) * grid - 1) / total);
+    if constexpr (k32) return static_cast<int>(((static_cast<uint32_t>(tile) + 1u) * static_cast<uint32_t>(grid) - 1u) / static_cast<uint32_t>(total));
+    else return static_cast<int>(((static_cast<long long>(tile) + 1) * grid - 1) / total);
 }
 
 // The chunks of a tile range [t0, t0 + ntiles): up to kR consecutive tiles of one strip each.  Tiles are stored
@@ -325,12 +334,12 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
     int cn = nclusters, crank = cta, cbase = 0, ctiles = total_tiles;
     if (CL && csize > 1) {
         const int q = cta / csize, strips = total_tiles / ktiles;
-        const int s0 = (int)(((long long)q * strips) / nclusters), s1 = (int)(((long long)(q + 1) * strips) / nclusters);
+        const int s0 = range_start<MT == 2>(q, strips, nclusters), s1 = range_start<MT == 2>(q + 1, strips, nclusters);
         cn = csize; crank = cta - q * csize; cbase = s0 * ktiles; ctiles = (s1 - s0) * ktiles;
     }
     const bool idle = crank >= cn;
-    const int t0 = idle ? 0 : cbase + range_start(crank, ctiles, cn);
-    const int ntiles = idle ? 0 : cbase + range_start(crank + 1, ctiles, cn) - t0;
+    const int t0 = idle ? 0 : cbase + range_start<MT == 2>(crank, ctiles, cn);
+    const int ntiles = idle ? 0 : cbase + range_start<MT == 2>(crank + 1, ctiles, cn) - t0;
     int fin_strip = -1, fin_first = 0;          // cluster mode: the strip this CTA finishes after the cluster barrier
 
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
@@ -411,8 +420,8 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
                 const int strip = tile0 / ktiles, T0 = tile0 - strip * ktiles;
                 const int seg_len = min(ntiles - i, ktiles - T0);
                 const bool whole = seg_len == ktiles;
-                const int c_first = range_owner(strip * ktiles - cbase, ctiles, cn);
-                const int c_last = range_owner(strip * ktiles + ktiles - 1 - cbase, ctiles, cn);
+                const int c_first = range_owner<MT == 2>(strip * ktiles - cbase, ctiles, cn);
+                const int c_last = range_owner<MT == 2>(strip * ktiles + ktiles - 1 - cbase, ctiles, cn);
                 // Global mode, cut strip: the CTA that holds the strip's first tile finishes it.  Its part of the strip
                 // is the tail of its range; for every other contributor the strip is the head of the range, done early.
                 const bool finisher = (!CL || csize == 1) && !whole && c_first == crank;
@@ -907,8 +916,12 @@ gemv_stream_kernel(const uint8_t* __restrict__ blob, const __nv_bfloat16* __rest
             float4 tot[kVec];
 #pragma unroll
             for (int e = 0; e < kVec; ++e) tot[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+            // (a range can be empty only where the cluster has fewer tiles than CTAs: the divisions of
+            // range_start stay out of this loop, which is the tail of the kernel, in every other case)
+            const bool some_empty = ctiles < cn;
+#pragma unroll 2
             for (int c = fin_first; c <= crank; ++c) {                     // rank order, as in global mode
-                if (range_start(c + 1, ctiles, cn) == range_start(c, ctiles, cn)) continue;   // empty range: no partial
+                if (some_empty && range_start<MT == 2>(c + 1, ctiles, cn) == range_start<MT == 2>(c, ctiles, cn)) continue;   // empty range: no partial
                 const float4* src = reinterpret_cast<const float4*>(xred + (size_t)c * xslot_bytes) + lane;
 #pragma unroll
                 for (int e = 0; e < kVec; ++e)
