@@ -17,16 +17,17 @@ namespace tf {
 // Configurations, chosen by plan_gemv:
 //   integer path (1 and 2 tokens), short ranges: 8 consumer warps and half an SM per CTA, so the next GEMV's CTAs
 //     fit beside this one's and have their rings full of weights when this kernel completes.
-//   integer path, long ranges: the whole SM, a ring of seven to ten stages, and as many consumer warps as hold
-//     about 66 KB of tiles (16 on 4-bit tiles, 8 on int8 tiles).
-//   Either form: where a range passes over its k-tiles more than once and K is a multiple of 128 x consumer warps,
-//     a warp keeps the activation pieces of the k-tiles it has visited (piece table) instead of preparing them per tile.
-//   floating-point path up to 8 tokens: the whole SM, 12 consumer warps and a ring deep enough to keep HBM busy
-//     while 12 tiles are being consumed.  A consumer warp
-//     of the floating-point path is bound by instruction issue (about 20 issue cycles per packed word of 8
-//     weights, measured on registers alone), and since a GEMV may not read its activations before the kernel ahead
-//     of it has completed, only one kernel's consumers work on an SM at a time: three warps per scheduler beat two
-//     warps plus a waiting neighbour (decode step of the benchmark: 133 against 140 us).
+//   integer path, long ranges: the whole SM, a ring of eight stages, and as many consumer warps as hold about
+//     66 KB of tiles (16 on 4-bit tiles, 8 on int8 tiles).
+//   Either form, 4-bit tiles: where a range passes over its k-tiles more than once and K is a multiple of 128 x
+//     consumer warps, a warp keeps the activation pieces of the k-tiles it has visited (piece table) instead of
+//     preparing them per tile.
+//   floating-point path up to 8 tokens: the whole SM and 12 consumer warps; on 4-bit tiles a ring of five stages
+//     (three in the warps' hands, two in flight; deeper was measured slower), on int8 tiles the deepest that fits.
+//     A consumer warp of the floating-point path is bound by instruction issue (about 20 issue cycles per packed
+//     word of 8 weights, measured on registers alone), and since a GEMV may not read its activations before the
+//     kernel ahead of it has completed, only one kernel's consumers work on an SM at a time: three warps per
+//     scheduler beat two warps plus a waiting neighbour (decode step of the benchmark: 133 against 140 us).
 //   9..16 tokens: twice the MMA and activation work per tile and the whole SM, but 8 consumer warps: every tile a
 //     warp is working on is a tile that is not in flight (measured on the four layer shapes with the ring holding
 //     weights only: 8 warps 7.9 / 4.1 / 14.5 / 15.4 us, 10 warps 8.4 / 4.1 / 15.2 / 16.1 us; 12 warps do not fit the
