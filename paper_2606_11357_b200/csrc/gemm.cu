@@ -50,6 +50,7 @@ constexpr int kTmemAccCols = 256;
 constexpr int kTmemCols = 512;
 constexpr int kMaxActStages = 12;
 constexpr int kWpStages = 3;              // packed-weight ring (one stage = the two strip tiles of one k-tile)
+static_assert(kWpStages <= kMaxDepth, "the barrier set-up gives one thread to each of kMaxDepth stages");
 
 // one packed tile of the ring, rounded up to a multiple of 128 bytes (G = groups per tile: 4256, 4416 or 4736 bytes of tile)
 __host__ __device__ constexpr int wp_strip_bytes(int bits, int G = 1) { return bits == 4 ? (G == 1 ? 4352 : G == 2 ? 4480 : 4736) : 8320; }
@@ -86,11 +87,13 @@ static_assert(kGemmCounterOffset + 4 * kGemmMaxTiles == kWorkspaceHeadBytes && k
               "workspace layout shared with the GEMV");
 constexpr int kGemmMaxGrid = 160;
 
+// 32-bit arithmetic: at most 256 x 16 x 256 units (N, K <= 32768, M <= 4096) times at most 161 CTAs stays below 2^28,
+// and these divisions sit between the start of a CTA and its first copy.
 __device__ __forceinline__ int unit_start(int cta, int total, int grid) {
-    return static_cast<int>((static_cast<long long>(cta) * total) / grid);
+    return static_cast<int>((static_cast<uint32_t>(cta) * static_cast<uint32_t>(total)) / static_cast<uint32_t>(grid));
 }
 __device__ __forceinline__ int unit_owner(int unit, int total, int grid) {
-    return static_cast<int>(((static_cast<long long>(unit) + 1) * grid - 1) / total);
+    return static_cast<int>(((static_cast<uint32_t>(unit) + 1u) * static_cast<uint32_t>(grid) - 1u) / static_cast<uint32_t>(total));
 }
 
 // The CTA's unit range [u_begin, u_end) as segments of one output tile each, in processing order: the cut tile at
@@ -223,15 +226,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap act_map, const uint8_t* __restri
     const bool header_ok = header_matches(blob, BITS, (uint32_t)K, (uint32_t)N) && group_size_fits(blob, G);
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(workspace);
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+    // (one thread per pipeline stage and one for the rest: the set-up sits between the start of a CTA and its first copy)
+    if (threadIdx.x < kMaxDepth) {
+        const int s = threadIdx.x;
+        if (s < kStages) {
             mbar_init(smem_u32(&bars->stage_full[s]), 9);    // eight dequant warps + the activation producer (with the bytes)
             mbar_init(smem_u32(&bars->stage_done[s]), 1);    // tcgen05.commit
         }
-        for (int s = 0; s < kWpStages; ++s) {
+        if (s < kWpStages) {
             mbar_init(smem_u32(&bars->wp_full[s]), 1);
             mbar_init(smem_u32(&bars->wp_empty[s]), 8);      // all eight dequant warps
         }
+        mbar_init_fence();
+    } else if (threadIdx.x == 32) {
         mbar_init(smem_u32(&bars->acc_full), 1);
         mbar_init(smem_u32(&bars->acc_empty), 12);           // four epilogue warps + eight dequant warps (drain duty)
         bars->abort_flag = 0;
