@@ -150,3 +150,16 @@ def test_config4_w4_gemm_k32768():
 def test_max_m_ragged():
     p = wl.make_w4(4096, 256, 200, seed=3)
     gu.check_against_oracle(p, gu.run(p, "gemm"))
+
+
+def test_maximum_dimensions_on_sampled_columns():
+    """M = 4096, K = N = 32768: the largest problem the GEMM accepts (256 x 16 tiles of 256 k-tiles each, split evenly
+    over the SMs), checked against the oracle on 129 sampled columns.  Codes drawn as whole words: uniform, as in make_w4."""
+    M, K, N = 4096, 32768, 32768
+    rng = np.random.default_rng(4343)
+    p = wl.Problem("w4max", 4, M, K, N, 128, 4343, wl._activations(rng, M, K),
+                   rng.uniform(0.001, 0.02, size=(K // 128, N)).astype(np.float32).astype(np.float16),
+                   qweight=rng.integers(0, 2**32, size=(K, N // 8), dtype=np.uint32),
+                   qzeros=rng.integers(0, 2**32, size=(K // 128, N // 8), dtype=np.uint32))
+    cols = np.unique(np.concatenate([np.arange(0, N, 257), [N - 1]]))
+    gu.check_against_oracle(p, gu.run(p, "gemm"), columns=cols)

@@ -1,4 +1,6 @@
 """Parity of tf_gemv_w4a16 / tf_gemv_w8a16 with the fp64 oracle, element by element."""
+import copy
+
 import numpy as np
 import pytest
 import torch
@@ -189,3 +191,23 @@ def test_config4_w4_gemv_32k_columns():
 def test_max_k_gemv():
     p = wl.make_w4(2, 32768, 128, seed=44)
     gu.check_against_oracle(p, gu.run(p, "gemv"))
+
+
+def test_maximum_dimensions_on_sampled_columns():
+    """K = N = 32768, the largest shape the library accepts (131072 tiles, a 558 MB blob): one token (integer path,
+    whole SM, piece table) and sixteen, checked against the oracle on 257 sampled columns (first, last and a stride
+    that meets every column position of a strip).  The codes are drawn as whole 32-bit words: uniform codes, like
+    make_w4's, at a fraction of the time."""
+    K = N = 32768
+    rng = np.random.default_rng(4242)
+    p = wl.Problem("w4max", 4, 16, K, N, 128, 4242, wl._activations(rng, 16, K),
+                   rng.uniform(0.001, 0.02, size=(K // 128, N)).astype(np.float32).astype(np.float16),
+                   qweight=rng.integers(0, 2**32, size=(K, N // 8), dtype=np.uint32),
+                   qzeros=rng.integers(0, 2**32, size=(K // 128, N // 8), dtype=np.uint32))
+    blob = torch.from_numpy(gu.pack(p)).cuda()
+    cols = np.unique(np.concatenate([np.arange(0, N, 129), [N - 1]]))
+    for M in (16, 1):
+        q = copy.copy(p)
+        q.M, q.a_bf16 = M, p.a_bf16[:M].copy()
+        y = gu.run(q, "gemv", blob_dev=blob)
+        gu.check_against_oracle(q, y, columns=cols)
