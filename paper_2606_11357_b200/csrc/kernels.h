@@ -43,8 +43,8 @@ constexpr int kGemvSoloSmemBytes = 114 * 1024;
 constexpr int kGemvPieceEntryBytes = 512;
 // Packed bytes per CTA from which the integer path uses the whole-SM configuration, and its consumer warps there.
 // A half-SM CTA has a ring of four or five 17 KB stages, and every tile a warp works on is a tile that is not in flight: eight
-// warps on int8 tiles (8.3 KB) hold the whole ring, on 4-bit tiles half of it.  The whole-SM form has a ring of nine
-// or ten stages; with about 66 KB of tiles in the warps' hands (8 warps on int8, 16 on 4-bit tiles) it streams long
+// warps on int8 tiles (8.3 KB) hold nearly the whole ring, on 4-bit tiles half of it.  The whole-SM form has a ring of
+// eight stages; with about 66 KB of tiles in the warps' hands (8 warps on int8, 16 on 4-bit tiles) it streams long
 // ranges faster than the half-SM form, which wins on short ranges because the next GEMV's CTAs sit beside it with
 // their rings full.
 constexpr int kGemvFullFromBytesI8W4 = TF_I8_FULL_BYTES_W4;
